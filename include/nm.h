@@ -1,0 +1,209 @@
+/*
+ * nm.h — C ABI of the column-wise N:M sparse convolution library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference hot path of "Efficient Column-Wise N:M Pruning on
+ * RISC-V CPU" (arXiv 2507.17301) on one GPU:
+ *
+ *   nm_prune      column-wise N:M pruning at tile level (Sec. 3.1) into the compressed
+ *                 weight + index-array form (Sec. 2.1, inputs of Algorithm 1);
+ *   nm_conv2d     convolution with those weights as a sparse implicit GEMM: the fused
+ *                 im2col + packing pass (Sec. 3.2, Algorithm 2) becomes an index-driven gather
+ *                 of the retained (kh, kw, c) slices from NHWC activations into shared memory,
+ *                 and the tiled outer-product micro-kernel (Algorithm 1) becomes a dense TF32
+ *                 tensor-core sub-GEMM per output-channel tile with fp32 accumulation;
+ *   nm_autotune   on-device profiling of candidate launch plans, keeping the fastest
+ *                 (Sec. 3.3).
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, fp32 unless stated,
+ *     contiguous, 16-byte aligned.  The library never frees or reallocates caller memory.
+ *     Entry points whose name ends in _host take HOST pointers instead and say so.
+ *   - Activations are NHWC  x[batch][h][w][c_in];  outputs NHWC  y[batch][ho][wo][c_out] with
+ *       ho = (h + 2*pad_h - dil_h*(kh-1) - 1) / stride_h + 1   (floor; same for wo).
+ *   - Dense weights are OHWI  w[c_out][kh][kw][c_in]; reduction column k = (kh*Kw + kw)*c_in + c
+ *     (Fig. 4: kernel layout OHWI), K = kh*kw*c_in <= 65535.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work
+ *     is enqueued on it; calls return without synchronising unless stated.
+ *   - All functions return an nm_status_t; nothing throws, aborts or exits.  A human-readable
+ *     description of the calling thread's last failure is available from nm_last_error().
+ *   - Handles (nm_weights_t) are owned by the library and released only by nm_weights_free.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point fails with
+ *     NM_ERR_CUDA.
+ */
+#ifndef NM_H_
+#define NM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NM_OK = 0,
+    NM_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, N > M, misaligned pointer, ... */
+    NM_ERR_UNSUPPORTED = -2, /* valid but outside what the kernels cover (K > 65535, tile > 256, ...) */
+    NM_ERR_CUDA = -3,        /* a CUDA runtime / driver call failed (text in nm_last_error) */
+    NM_ERR_ALLOC = -4,       /* host or device allocation failed */
+    NM_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported by nm_weights_check) */
+    NM_ERR_INTERNAL = -6
+} nm_status_t;
+
+/* Opaque compressed-weight handle: compacted values, per-tile column indices and the
+ * library's internal copies (TF32-rounded, padded weight tiles; decoded tap table). */
+typedef struct nm_weights nm_weights_t;
+
+/*
+ * Launch plan for nm_conv2d (the analogue of the paper's per-layer template parameters, Sec. 3.3).
+ *   variant  0 = let the library choose; 1 = direct-gather kernel (any shape);
+ *            2 = slab kernel (dense activation slab staged once per CTA, compacted on chip;
+ *                needs c_in % 4 == 0 and m_group | 32-column slab, see nm_conv2d)
+ *   bn       output channels per CTA (a multiple of the weights' tile_t), 0 = default
+ *   stages   depth of the shared-memory ring, 0 = default
+ *   split    reserved, 0
+ */
+typedef struct {
+    int variant;
+    int bn;
+    int stages;
+    int split;
+    int reserved[12];
+} nm_plan_t;
+
+/* ---------------------------------------------------------------------------------------------
+ * Pruning and the compressed form
+ * ------------------------------------------------------------------------------------------- */
+
+/*
+ * Column-wise N:M pruning at tile level (Sec. 3.1).
+ * Rows of the [c_out, K] filter matrix are cut into tiles of `tile_t` output channels.  Inside a
+ * tile a column (its tile_t weights) is one unit scored by its L1 norm; in every group of
+ * `m_group` consecutive columns the `n_keep` highest-scoring units are RETAINED (N counts kept
+ * columns: "N = (1 - sparsity) * M") and all rows of the tile share that kept set.
+ * Deterministic rules where the paper is silent: scores are fp64 sums over the tile's rows in
+ * ascending row order; of two equal scores the lower column is kept; a tail group of m' < M
+ * columns keeps min(N, m'); a tail tile (c_out % tile_t rows) scores over the rows it has.
+ *
+ *   w_dense   device, fp32 [c_out][kh][kw][c_in]; read only, may be freed after the stream
+ *             has passed this call
+ *   out       receives a new handle holding values[c_out][kk] and indices[n_tiles][kk]
+ *             (see nm_weights_export) with kk = N*(K / M) + min(N, K % M)
+ * Allocates device memory (synchronously); the kernels run on `cuda_stream`.
+ * Errors: INVALID_ARG (null, sizes < 1, n_keep > m_group), UNSUPPORTED (K > 65535, kh or kw > 255,
+ * tile_t > 256), ALLOC, CUDA.
+ */
+nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep,
+                     int m_group, int tile_t, void* cuda_stream, nm_weights_t** out);
+
+/* Dimensions of a handle; any output pointer may be NULL. */
+nm_status_t nm_weights_dims(const nm_weights_t* w, int* c_out, int* k, int* kk, int* n_tiles,
+                            int* tile_t);
+
+/*
+ * Copies the canonical compressed form (Sec. 2.1: "a compressed weight format and an index
+ * array"; Algorithm 1 inputs W[T, N] and Idx[N]) to caller memory on `cuda_stream`:
+ *   values   device, fp32 [c_out][kk]: values[o][j] = w[o][indices[o / tile_t][j]], bit-exact
+ *   indices  device, uint16 [n_tiles][kk]: absolute column positions k, ascending
+ * Either pointer may be NULL to skip it.
+ */
+nm_status_t nm_weights_export(const nm_weights_t* w, float* values, uint16_t* indices,
+                              void* cuda_stream);
+
+/*
+ * Builds a handle from an already compressed model (the inverse of nm_weights_export; this is the
+ * checkpoint path).  Validates on the device that every index row is strictly ascending and
+ * < K; the group structure is not re-checked.  Same errors as nm_prune, plus INVALID_ARG for a bad
+ * index row (detected synchronously).
+ */
+nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int c_out, int kh,
+                              int kw, int c_in, int n_keep, int m_group, int tile_t,
+                              void* cuda_stream, nm_weights_t** out);
+
+/* Synchronises `cuda_stream`, then reads the handle's device status word.  Returns NM_OK, or
+ * NM_ERR_TIMEOUT if a kernel that used this handle gave up on a bounded wait (the status word is
+ * cleared, the context stays usable). */
+nm_status_t nm_weights_check(const nm_weights_t* w, void* cuda_stream);
+
+/* Releases the handle and its device memory (synchronises the device first). NULL is accepted. */
+nm_status_t nm_weights_free(nm_weights_t* w);
+
+/* ---------------------------------------------------------------------------------------------
+ * Convolution
+ * ------------------------------------------------------------------------------------------- */
+
+/*
+ * y = act(conv(x, W_pruned) + bias): the product of Algorithm 1 taken over the patch matrix of
+ * Sec. 2.2, which is never materialised: for each output-channel tile only the retained
+ * (kh, kw, c) slices are gathered (Sec. 3.2's fused im2col + packing, done as a gathered load).
+ *   y[n][oh][ow][o] = act( bias[o] + sum_j values[o][j] *
+ *                          x[n][oh*stride_h - pad_h + kh_j*dil_h][ow*stride_w - pad_w + kw_j*dil_w][c_j] )
+ * with (kh_j, kw_j, c_j) decoded from indices[o / tile_t][j] and reads outside the image = 0.
+ * Arithmetic: operands rounded to TF32 (weights once at prune time, round-to-nearest; activations
+ * round-to-nearest where they pass through registers, truncated where the staged slab feeds the
+ * tensor core directly), products accumulated in fp32.
+ *
+ *   x      device fp32 [batch][h][wd][c_in]      bias  device fp32 [c_out] or NULL
+ *   y      device fp32 [batch][ho][wo][c_out]    relu  0 = identity, 1 = ReLU
+ *   plan   NULL = library default; a plan the shape does not admit gives NM_ERR_UNSUPPORTED
+ * Asynchronous on `cuda_stream`; allocates nothing.  Errors: INVALID_ARG (null x / y / w, sizes,
+ * no output pixels, misaligned pointers), UNSUPPORTED, CUDA (launch failure).
+ */
+nm_status_t nm_conv2d(const nm_weights_t* w, const float* x, int batch, int h, int wd,
+                      int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                      const float* bias, int relu, float* y, const nm_plan_t* plan,
+                      void* cuda_stream);
+
+/*
+ * Same operation with HOST buffers: x_host, bias_host and y_host are host pointers (pinned memory
+ * makes the copies asynchronous), x_dev / y_dev are caller-owned device staging buffers of the
+ * sizes nm_conv2d expects and bias_dev a device buffer of c_out floats (may be NULL iff bias_host
+ * is).  Enqueues H2D(x, bias) -> nm_conv2d -> D2H(y) on `cuda_stream`; does not synchronise.
+ */
+nm_status_t nm_conv2d_host(const nm_weights_t* w, const float* x_host, float* x_dev, int batch,
+                           int h, int wd, int stride_h, int stride_w, int pad_h, int pad_w,
+                           int dil_h, int dil_w, const float* bias_host, float* bias_dev, int relu,
+                           float* y_host, float* y_dev, const nm_plan_t* plan, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Auto-tuning (Sec. 3.3: profile kernel candidates on the target, keep the fastest)
+ * ------------------------------------------------------------------------------------------- */
+
+/*
+ * Times every launch plan the library admits for this layer (kernel variant x channels per CTA x
+ * ring depth) with CUDA events on `cuda_stream` (a few warm-up launches, then the median of
+ * several), writes the fastest to *best and its time to *best_ms (may be NULL).  x and y_scratch
+ * are caller buffers of the sizes nm_conv2d expects; y_scratch is overwritten.  Synchronises the
+ * stream.  A candidate that fails to launch is skipped; NM_ERR_UNSUPPORTED if none runs.
+ */
+nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h, int wd,
+                        int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                        const float* bias, int relu, float* y_scratch, void* cuda_stream,
+                        nm_plan_t* best, float* best_ms);
+
+/*
+ * Auto-tuning that also chooses the pruning tile width T (the paper profiles T per layer,
+ * Sec. 3.3 / Sec. 4.5): prunes `w_dense` once per entry of tile_candidates, tunes each with
+ * nm_autotune and returns the fastest (tile, plan) pair.  *best_tile receives the chosen T.
+ * The handles it builds are temporary and freed before returning.
+ */
+nm_status_t nm_autotune_tile(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep,
+                             int m_group, const int* tile_candidates, int n_candidates,
+                             const float* x, int batch, int h, int wd, int stride_h, int stride_w,
+                             int pad_h, int pad_w, int dil_h, int dil_w, const float* bias, int relu,
+                             float* y_scratch, void* cuda_stream, int* best_tile, nm_plan_t* best,
+                             float* best_ms);
+
+/* ---------------------------------------------------------------------------------------------
+ * Diagnostics
+ * ------------------------------------------------------------------------------------------- */
+
+const char* nm_status_string(nm_status_t s);
+/* Text of the calling thread's most recent failure ("" if none). Valid until its next failure. */
+const char* nm_last_error(void);
+/* Number of kernel launches this process has enqueued through the library (all threads). */
+uint64_t nm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NM_H_ */

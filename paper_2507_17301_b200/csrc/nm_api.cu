@@ -1,0 +1,372 @@
+// Host side of the C ABI declared in include/nm.h: argument checks, handle life cycle, plan
+// resolution, launches, auto-tuning.  No tensor type other than raw pointers crosses this file.
+#include <algorithm>
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "nm_internal.h"
+
+namespace {
+thread_local char g_err[512] = "";
+std::atomic<uint64_t> g_launches{0};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int kept_count(int k, int n_keep, int m_group)
+{
+    const int full = k / m_group, tail = k % m_group;
+    return full * n_keep + std::min(tail, n_keep);
+}
+
+void free_handle_memory(nm_weights* h)
+{
+    if (!h) return;
+    cudaFree(h->values);
+    cudaFree(h->indices);
+    cudaFree(h->wt);
+    cudaFree(h->taps);
+    cudaFree(h->status);
+    h->magic = 0;
+    delete h;
+}
+
+// Validates the layer description and allocates an empty handle.
+nm_status_t make_handle(const char* who, int c_out, int kh, int kw, int c_in, int n_keep, int m_group, int tile_t,
+                        nm_weights** out)
+{
+    if (!out) return nmhost::fail(NM_ERR_INVALID_ARG, "%s: out is NULL", who);
+    *out = nullptr;
+    if (c_out < 1 || kh < 1 || kw < 1 || c_in < 1)
+        return nmhost::fail(NM_ERR_INVALID_ARG, "%s: c_out, kh, kw, c_in must be >= 1", who);
+    if (n_keep < 1 || m_group < 1 || n_keep > m_group)
+        return nmhost::fail(NM_ERR_INVALID_ARG, "%s: need 1 <= n_keep <= m_group (got %d:%d)", who, n_keep, m_group);
+    if (tile_t < 1) return nmhost::fail(NM_ERR_INVALID_ARG, "%s: tile_t must be >= 1", who);
+    const long long k = static_cast<long long>(kh) * kw * c_in;
+    if (k > 65535) return nmhost::fail(NM_ERR_UNSUPPORTED, "%s: K = %lld exceeds the uint16 index range", who, k);
+    if (kh > 255 || kw > 255) return nmhost::fail(NM_ERR_UNSUPPORTED, "%s: kernel extent above 255", who);
+    if (tile_t > 256) return nmhost::fail(NM_ERR_UNSUPPORTED, "%s: tile_t above 256", who);
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "%s: cudaGetDevice: %s", who, cudaGetErrorString(e));
+
+    nm_weights* h = new (std::nothrow) nm_weights();
+    if (!h) return nmhost::fail(NM_ERR_ALLOC, "%s: out of host memory", who);
+    std::memset(h, 0, sizeof(*h));
+    h->magic = NM_MAGIC;
+    h->device = dev;
+    h->c_out = c_out; h->kh = kh; h->kw = kw; h->c_in = c_in;
+    h->k = static_cast<int>(k);
+    h->n_keep = n_keep; h->m_group = m_group; h->tile_t = tile_t;
+    h->kk = kept_count(h->k, n_keep, m_group);
+    h->n_tiles = (c_out + tile_t - 1) / tile_t;
+    h->kk_pad = ((h->kk + NM_KCHUNK - 1) / NM_KCHUNK) * NM_KCHUNK;
+    const size_t nv = static_cast<size_t>(c_out) * std::max(h->kk, 1);
+    const size_t ni = static_cast<size_t>(h->n_tiles) * std::max(h->kk, 1);
+    const size_t nw = static_cast<size_t>(c_out) * h->kk_pad;
+    const size_t nt = static_cast<size_t>(h->n_tiles) * h->kk_pad;
+    if (cudaMalloc(&h->values, nv * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&h->indices, ni * sizeof(uint16_t)) != cudaSuccess ||
+        cudaMalloc(&h->wt, std::max<size_t>(nw, 1) * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&h->taps, std::max<size_t>(nt, 1) * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMalloc(&h->status, 4 * sizeof(int)) != cudaSuccess || cudaMemset(h->status, 0, 4 * sizeof(int)) != cudaSuccess) {
+        const char* msg = cudaGetErrorString(cudaGetLastError());
+        free_handle_memory(h);
+        return nmhost::fail(NM_ERR_ALLOC, "%s: device allocation failed: %s", who, msg);
+    }
+    *out = h;
+    return NM_OK;
+}
+
+bool valid(const nm_weights* w) { return w && w->magic == NM_MAGIC; }
+
+// Checks a conv call and fills the kernel parameters.
+nm_status_t make_params(const char* who, const nm_weights* w, const float* x, int batch, int h, int wd, int stride_h,
+                        int stride_w, int pad_h, int pad_w, int dil_h, int dil_w, const float* bias, int relu,
+                        float* y, ConvParams* p)
+{
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "%s: bad weights handle", who);
+    if (!x || !y) return nmhost::fail(NM_ERR_INVALID_ARG, "%s: x or y is NULL", who);
+    if (batch < 1 || h < 1 || wd < 1) return nmhost::fail(NM_ERR_INVALID_ARG, "%s: batch, h, w must be >= 1", who);
+    if (stride_h < 1 || stride_w < 1 || dil_h < 1 || dil_w < 1 || pad_h < 0 || pad_w < 0)
+        return nmhost::fail(NM_ERR_INVALID_ARG, "%s: stride and dilation must be >= 1, padding >= 0", who);
+    if (!aligned16(x) || !aligned16(y) || (bias && !aligned16(bias)))
+        return nmhost::fail(NM_ERR_INVALID_ARG, "%s: x, y and bias must be 16-byte aligned", who);
+    const long long eh = static_cast<long long>(h) + 2ll * pad_h - static_cast<long long>(dil_h) * (w->kh - 1) - 1;
+    const long long ew = static_cast<long long>(wd) + 2ll * pad_w - static_cast<long long>(dil_w) * (w->kw - 1) - 1;
+    if (eh < 0 || ew < 0) return nmhost::fail(NM_ERR_INVALID_ARG, "%s: the kernel does not fit the padded image", who);
+    const long long ho = eh / stride_h + 1, wo = ew / stride_w + 1;
+    const long long pixels = static_cast<long long>(batch) * ho * wo;
+    if (ho > 0x7FFFFFFF || wo > 0x7FFFFFFF || pixels > (1ll << 40))
+        return nmhost::fail(NM_ERR_UNSUPPORTED, "%s: output too large", who);
+    p->x = x; p->wt = w->wt; p->taps = w->taps; p->bias = bias; p->y = y; p->status = w->status;
+    p->batch = batch; p->h = h; p->w = wd; p->c_in = w->c_in;
+    p->ho = static_cast<int>(ho); p->wo = static_cast<int>(wo); p->c_out = w->c_out;
+    p->stride_h = stride_h; p->stride_w = stride_w; p->pad_h = pad_h; p->pad_w = pad_w;
+    p->dil_h = dil_h; p->dil_w = dil_w; p->kh = w->kh; p->kw = w->kw;
+    p->kk = w->kk; p->kk_pad = w->kk_pad; p->tile_t = w->tile_t; p->n_tiles = w->n_tiles; p->relu = relu ? 1 : 0;
+    p->n_keep = w->n_keep; p->m_group = w->m_group;
+    p->pixels = pixels;
+    return NM_OK;
+}
+
+nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st)
+{
+    const int variant = plan ? plan->variant : 0;
+    switch (variant) {
+        case 0:
+        case 1:
+            return nmhost::launch_conv_gather(p, st);
+        default:
+            return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
+    }
+}
+
+// Candidate plans for a layer, most promising first.
+std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams& /*p*/)
+{
+    std::vector<nm_plan_t> out;
+    nm_plan_t a;
+    std::memset(&a, 0, sizeof(a));
+    a.variant = 1;
+    out.push_back(a);
+    return out;
+}
+
+}  // namespace
+
+namespace nmhost {
+nm_status_t fail(nm_status_t s, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+}  // namespace nmhost
+
+extern "C" {
+
+nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep, int m_group, int tile_t,
+                     void* cuda_stream, nm_weights_t** out)
+{
+    if (!w_dense) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_prune: w_dense is NULL");
+    nm_weights* h = nullptr;
+    nm_status_t s = make_handle("nm_prune", c_out, kh, kw, c_in, n_keep, m_group, tile_t, &h);
+    if (s != NM_OK) return s;
+    s = nmhost::prune_on_device(w_dense, h, static_cast<cudaStream_t>(cuda_stream));
+    if (s != NM_OK) {
+        free_handle_memory(h);
+        return s;
+    }
+    *out = h;
+    return NM_OK;
+}
+
+nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int c_out, int kh, int kw, int c_in,
+                              int n_keep, int m_group, int tile_t, void* cuda_stream, nm_weights_t** out)
+{
+    if (!values || !indices) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_import: values or indices is NULL");
+    nm_weights* h = nullptr;
+    nm_status_t s = make_handle("nm_weights_import", c_out, kh, kw, c_in, n_keep, m_group, tile_t, &h);
+    if (s != NM_OK) return s;
+    s = nmhost::build_from_compressed(values, indices, h, static_cast<cudaStream_t>(cuda_stream));
+    if (s != NM_OK) {
+        free_handle_memory(h);
+        *out = nullptr;
+        return s;
+    }
+    *out = h;
+    return NM_OK;
+}
+
+nm_status_t nm_weights_dims(const nm_weights_t* w, int* c_out, int* k, int* kk, int* n_tiles, int* tile_t)
+{
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_dims: bad weights handle");
+    if (c_out) *c_out = w->c_out;
+    if (k) *k = w->k;
+    if (kk) *kk = w->kk;
+    if (n_tiles) *n_tiles = w->n_tiles;
+    if (tile_t) *tile_t = w->tile_t;
+    return NM_OK;
+}
+
+nm_status_t nm_weights_export(const nm_weights_t* w, float* values, uint16_t* indices, void* cuda_stream)
+{
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_export: bad weights handle");
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaSuccess;
+    if (values && w->kk > 0)
+        e = cudaMemcpyAsync(values, w->values, static_cast<size_t>(w->c_out) * w->kk * sizeof(float),
+                            cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess && indices && w->kk > 0)
+        e = cudaMemcpyAsync(indices, w->indices, static_cast<size_t>(w->n_tiles) * w->kk * sizeof(uint16_t),
+                            cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_weights_export: %s", cudaGetErrorString(e));
+    return NM_OK;
+}
+
+nm_status_t nm_weights_check(const nm_weights_t* w, void* cuda_stream)
+{
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_check: bad weights handle");
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int host[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaMemcpyAsync(host, w->status, sizeof(host), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_weights_check: %s", cudaGetErrorString(e));
+    if (host[0] != 0) {
+        cudaMemsetAsync(w->status, 0, 3 * sizeof(int), st);
+        cudaStreamSynchronize(st);
+        return nmhost::fail(static_cast<nm_status_t>(host[0]), "device-side wait expired (site %d, block %d)", host[1],
+                            host[2]);
+    }
+    return NM_OK;
+}
+
+nm_status_t nm_weights_free(nm_weights_t* w)
+{
+    if (!w) return NM_OK;
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_free: bad weights handle");
+    cudaDeviceSynchronize();
+    free_handle_memory(w);
+    return NM_OK;
+}
+
+nm_status_t nm_conv2d(const nm_weights_t* w, const float* x, int batch, int h, int wd, int stride_h, int stride_w,
+                      int pad_h, int pad_w, int dil_h, int dil_w, const float* bias, int relu, float* y,
+                      const nm_plan_t* plan, void* cuda_stream)
+{
+    ConvParams p;
+    nm_status_t s = make_params("nm_conv2d", w, x, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, bias,
+                                relu, y, &p);
+    if (s != NM_OK) return s;
+    return run_plan(p, plan, static_cast<cudaStream_t>(cuda_stream));
+}
+
+nm_status_t nm_conv2d_host(const nm_weights_t* w, const float* x_host, float* x_dev, int batch, int h, int wd,
+                           int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                           const float* bias_host, float* bias_dev, int relu, float* y_host, float* y_dev,
+                           const nm_plan_t* plan, void* cuda_stream)
+{
+    if (!x_host || !y_host) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_conv2d_host: x_host or y_host is NULL");
+    if (bias_host && !bias_dev) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_conv2d_host: bias_dev is NULL");
+    ConvParams p;
+    nm_status_t s = make_params("nm_conv2d_host", w, x_dev, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h,
+                                dil_w, bias_host ? bias_dev : nullptr, relu, y_dev, &p);
+    if (s != NM_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t xb = static_cast<size_t>(batch) * h * wd * w->c_in * sizeof(float);
+    const size_t yb = static_cast<size_t>(p.pixels) * w->c_out * sizeof(float);
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && bias_host)
+        e = cudaMemcpyAsync(bias_dev, bias_host, static_cast<size_t>(w->c_out) * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_conv2d_host: H2D copy: %s", cudaGetErrorString(e));
+    s = run_plan(p, plan, st);
+    if (s != NM_OK) return s;
+    e = cudaMemcpyAsync(y_host, y_dev, yb, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_conv2d_host: D2H copy: %s", cudaGetErrorString(e));
+    return NM_OK;
+}
+
+nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h, int wd, int stride_h, int stride_w,
+                        int pad_h, int pad_w, int dil_h, int dil_w, const float* bias, int relu, float* y_scratch,
+                        void* cuda_stream, nm_plan_t* best, float* best_ms)
+{
+    if (!best) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_autotune: best is NULL");
+    ConvParams p;
+    nm_status_t s = make_params("nm_autotune", w, x, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                bias, relu, y_scratch, &p);
+    if (s != NM_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        return nmhost::fail(NM_ERR_CUDA, "nm_autotune: cannot create events");
+    }
+    constexpr int kWarm = 2, kReps = 7;
+    float best_t = -1.f;
+    for (const nm_plan_t& cand : candidate_plans(w, p)) {
+        bool ok = true;
+        for (int i = 0; i < kWarm && ok; ++i) ok = run_plan(p, &cand, st) == NM_OK;
+        if (!ok || cudaStreamSynchronize(st) != cudaSuccess) continue;
+        std::vector<float> t;
+        for (int i = 0; i < kReps && ok; ++i) {
+            cudaEventRecord(e0, st);
+            ok = run_plan(p, &cand, st) == NM_OK;
+            cudaEventRecord(e1, st);
+            if (cudaEventSynchronize(e1) != cudaSuccess) ok = false;
+            float ms = 0.f;
+            if (ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess) t.push_back(ms);
+        }
+        if (!ok || t.empty()) continue;
+        std::sort(t.begin(), t.end());
+        const float med = t[t.size() / 2];
+        if (best_t < 0.f || med < best_t) {
+            best_t = med;
+            *best = cand;
+        }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (best_t < 0.f) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_autotune: no candidate plan ran");
+    if (best_ms) *best_ms = best_t;
+    return nm_weights_check(w, cuda_stream);
+}
+
+nm_status_t nm_autotune_tile(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep, int m_group,
+                             const int* tile_candidates, int n_candidates, const float* x, int batch, int h, int wd,
+                             int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w, const float* bias,
+                             int relu, float* y_scratch, void* cuda_stream, int* best_tile, nm_plan_t* best,
+                             float* best_ms)
+{
+    if (!tile_candidates || n_candidates < 1 || !best_tile || !best)
+        return nmhost::fail(NM_ERR_INVALID_ARG, "nm_autotune_tile: candidates / outputs missing");
+    float best_t = -1.f;
+    nm_status_t last = NM_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_candidates; ++i) {
+        nm_weights_t* hnd = nullptr;
+        last = nm_prune(w_dense, c_out, kh, kw, c_in, n_keep, m_group, tile_candidates[i], cuda_stream, &hnd);
+        if (last != NM_OK) continue;
+        nm_plan_t plan;
+        float ms = 0.f;
+        last = nm_autotune(hnd, x, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, bias, relu, y_scratch,
+                           cuda_stream, &plan, &ms);
+        nm_weights_free(hnd);
+        if (last != NM_OK) continue;
+        if (best_t < 0.f || ms < best_t) {
+            best_t = ms;
+            *best_tile = tile_candidates[i];
+            *best = plan;
+        }
+    }
+    if (best_t < 0.f) return last == NM_OK ? nmhost::fail(NM_ERR_UNSUPPORTED, "nm_autotune_tile: nothing ran") : last;
+    if (best_ms) *best_ms = best_t;
+    return NM_OK;
+}
+
+const char* nm_status_string(nm_status_t s)
+{
+    switch (s) {
+        case NM_OK: return "NM_OK";
+        case NM_ERR_INVALID_ARG: return "NM_ERR_INVALID_ARG";
+        case NM_ERR_UNSUPPORTED: return "NM_ERR_UNSUPPORTED";
+        case NM_ERR_CUDA: return "NM_ERR_CUDA";
+        case NM_ERR_ALLOC: return "NM_ERR_ALLOC";
+        case NM_ERR_TIMEOUT: return "NM_ERR_TIMEOUT";
+        case NM_ERR_INTERNAL: return "NM_ERR_INTERNAL";
+    }
+    return "NM_ERR_UNKNOWN";
+}
+
+const char* nm_last_error(void) { return g_err; }
+
+uint64_t nm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

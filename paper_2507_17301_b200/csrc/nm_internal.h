@@ -1,0 +1,53 @@
+// Library-internal declarations shared by the host API and the kernel translation units.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/nm.h"
+
+constexpr uint32_t NM_MAGIC = 0x4E4D5754u;  // "NMWT"
+constexpr uint32_t NM_TAP_PAD = 0xFFFFFFFFu;  // tap-table entry of a padding column: gathers zero
+constexpr int NM_KCHUNK = 32;               // kept columns per shared-memory operand chunk (128 B of TF32)
+
+// Compressed weights of one layer.  `values` / `indices` are the canonical, exportable form;
+// `wt` and `taps` are what the convolution kernels read.
+struct nm_weights {
+    uint32_t magic;
+    int device;
+    int c_out, kh, kw, c_in, k, kk, n_keep, m_group, tile_t, n_tiles;
+    int kk_pad;          // kk rounded up to a multiple of NM_KCHUNK
+    float* values;       // [c_out][kk]     exact fp32 copies of the retained weights
+    uint16_t* indices;   // [n_tiles][kk]   retained column positions, ascending
+    float* wt;           // [c_out][kk_pad] retained weights rounded to TF32 (nearest), zero padded
+    uint32_t* taps;      // [n_tiles][kk_pad] kh << 24 | kw << 16 | c per retained column, NM_TAP_PAD in the padding
+    int* status;         // device int[4]: [0] error code, [1] where, [2] block, [3] spare
+};
+
+// Geometry handed to the convolution kernels.
+struct ConvParams {
+    const float* x;
+    const float* wt;
+    const uint32_t* taps;
+    const float* bias;
+    float* y;
+    int* status;
+    int batch, h, w, c_in, ho, wo, c_out;
+    int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+    int kh, kw;
+    int kk, kk_pad, tile_t, n_tiles, relu;
+    int n_keep, m_group;
+    long long pixels;  // batch * ho * wo
+};
+
+namespace nmhost {
+// Sets the calling thread's error text and returns `s`.
+nm_status_t fail(nm_status_t s, const char* fmt, ...);
+void count_launch(int n = 1);
+
+// nm_prune.cu
+nm_status_t prune_on_device(const float* w_dense, nm_weights* h, cudaStream_t st);
+nm_status_t build_from_compressed(const float* values, const uint16_t* indices, nm_weights* h, cudaStream_t st);
+
+// nm_conv_gather.cu — variant 1
+nm_status_t launch_conv_gather(const ConvParams& p, cudaStream_t st);
+}  // namespace nmhost

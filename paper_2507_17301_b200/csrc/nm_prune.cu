@@ -1,0 +1,187 @@
+// Column-wise N:M pruning at tile level (Sec. 3.1) on the device, and construction of the
+// kernel-side copies of the compressed form (Sec. 2.1; inputs W and Idx of Algorithm 1).
+//
+// Four small kernels, all one thread per (tile, column) or (row, retained column):
+//   score    s[r][k]   = sum over the tile's rows of |w[o][k]|, fp64, ascending row order
+//   select   keep[r][k] = 1 iff fewer than N columns of k's group beat it, where column i beats
+//            column k when s[i] > s[k], or s[i] == s[k] and i < k (lower column wins ties)
+//   compact  position of each kept column = N * group + number of kept columns before it in its
+//            group; writes the index array and the decoded (kh, kw, c) tap table
+//   gather   values[o][j] = w[o][idx[j]] (bit copy) and the TF32-rounded, zero-padded copy
+// The selection rule is the closed form of "pick the largest N times": both orderings are the
+// sort by (score descending, column ascending), so the result is unique and bit-reproducible as
+// long as the fp64 sums are formed in the same order everywhere.
+#include <cstdio>
+
+#include "nm_internal.h"
+#include "nm_ptx.cuh"
+
+namespace {
+
+__global__ void k_score(const float* __restrict__ w, int c_out, int k, int tile_t, double* __restrict__ score)
+{
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.y;
+    if (col >= k) return;
+    const int row0 = r * tile_t;
+    const int row1 = min(row0 + tile_t, c_out);
+    double s = 0.0;
+    for (int o = row0; o < row1; ++o) s += fabs(static_cast<double>(w[static_cast<size_t>(o) * k + col]));
+    score[static_cast<size_t>(r) * k + col] = s;
+}
+
+__global__ void k_select(const double* __restrict__ score, int k, int n_keep, int m_group,
+                         uint8_t* __restrict__ keep)
+{
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.y;
+    if (col >= k) return;
+    const double* s = score + static_cast<size_t>(r) * k;
+    const int g0 = (col / m_group) * m_group;
+    const int g1 = min(g0 + m_group, k);
+    const double mine = s[col];
+    int beaten_by = 0;
+    for (int i = g0; i < g1; ++i) {
+        const double si = s[i];
+        beaten_by += (si > mine) || (si == mine && i < col);
+    }
+    keep[static_cast<size_t>(r) * k + col] = beaten_by < n_keep ? 1 : 0;
+}
+
+__global__ void k_compact(const uint8_t* __restrict__ keep, int k, int kk, int kk_pad, int n_keep, int m_group,
+                          int c_in, int kw, uint16_t* __restrict__ indices, uint32_t* __restrict__ taps)
+{
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.y;
+    if (col >= k) return;
+    const uint8_t* kp = keep + static_cast<size_t>(r) * k;
+    if (!kp[col]) return;
+    const int g = col / m_group;
+    int pos = g * n_keep;  // every earlier group is a full one and kept exactly n_keep
+    for (int i = g * m_group; i < col; ++i) pos += kp[i];
+    indices[static_cast<size_t>(r) * kk + pos] = static_cast<uint16_t>(col);
+    const int c = col % c_in, tap = col / c_in;
+    taps[static_cast<size_t>(r) * kk_pad + pos] =
+        (static_cast<uint32_t>(tap / kw) << 24) | (static_cast<uint32_t>(tap % kw) << 16) | static_cast<uint32_t>(c);
+}
+
+// From indices alone (import path): tap table.
+__global__ void k_taps_from_indices(const uint16_t* __restrict__ indices, int kk, int kk_pad, int c_in, int kw,
+                                    uint32_t* __restrict__ taps)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.y;
+    if (j >= kk) return;
+    const int col = indices[static_cast<size_t>(r) * kk + j];
+    const int c = col % c_in, tap = col / c_in;
+    taps[static_cast<size_t>(r) * kk_pad + j] =
+        (static_cast<uint32_t>(tap / kw) << 24) | (static_cast<uint32_t>(tap % kw) << 16) | static_cast<uint32_t>(c);
+}
+
+__global__ void k_gather_values(const float* __restrict__ w, const uint16_t* __restrict__ indices, int k, int kk,
+                                int kk_pad, int tile_t, float* __restrict__ values, float* __restrict__ wt)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int o = blockIdx.y;
+    if (j >= kk_pad) return;
+    float v = 0.f;
+    if (j < kk) {
+        v = w[static_cast<size_t>(o) * k + indices[static_cast<size_t>(o / tile_t) * kk + j]];
+        values[static_cast<size_t>(o) * kk + j] = v;
+    }
+    wt[static_cast<size_t>(o) * kk_pad + j] = nmk::to_tf32(v);
+}
+
+// Import path: values already compacted.
+__global__ void k_round_values(const float* __restrict__ values, int kk, int kk_pad, float* __restrict__ wt)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int o = blockIdx.y;
+    if (j >= kk_pad) return;
+    const float v = j < kk ? values[static_cast<size_t>(o) * kk + j] : 0.f;
+    wt[static_cast<size_t>(o) * kk_pad + j] = nmk::to_tf32(v);
+}
+
+// Import path: every index row must be strictly ascending and below k.
+__global__ void k_check_indices(const uint16_t* __restrict__ indices, int kk, int k, int* __restrict__ bad)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.y;
+    if (j >= kk) return;
+    const int v = indices[static_cast<size_t>(r) * kk + j];
+    if (v >= k || (j > 0 && indices[static_cast<size_t>(r) * kk + j - 1] >= v)) atomicExch(bad, 1);
+}
+
+#define NM_CUDA_TRY(call)                                                                                   \
+    do {                                                                                                    \
+        cudaError_t e__ = (call);                                                                           \
+        if (e__ != cudaSuccess) {                                                                           \
+            st_out = nmhost::fail(NM_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e__));            \
+            goto done;                                                                                      \
+        }                                                                                                   \
+    } while (0)
+
+}  // namespace
+
+namespace nmhost {
+
+nm_status_t prune_on_device(const float* w_dense, nm_weights* h, cudaStream_t st)
+{
+    nm_status_t st_out = NM_OK;
+    double* score = nullptr;
+    uint8_t* keep = nullptr;
+    const size_t cells = static_cast<size_t>(h->n_tiles) * h->k;
+    const dim3 blk(128);
+    const dim3 grid_cols((h->k + 127) / 128, h->n_tiles);
+    const dim3 grid_vals((h->kk_pad + 127) / 128, h->c_out);
+
+    if (cudaMalloc(&score, cells * sizeof(double)) != cudaSuccess || cudaMalloc(&keep, cells) != cudaSuccess) {
+        (void)cudaGetLastError();
+        st_out = fail(NM_ERR_ALLOC, "nm_prune: cannot allocate %zu bytes of scratch", cells * 9);
+        goto done;
+    }
+    NM_CUDA_TRY(cudaMemsetAsync(h->taps, 0xFF, static_cast<size_t>(h->n_tiles) * h->kk_pad * sizeof(uint32_t), st));
+    k_score<<<grid_cols, blk, 0, st>>>(w_dense, h->c_out, h->k, h->tile_t, score);
+    k_select<<<grid_cols, blk, 0, st>>>(score, h->k, h->n_keep, h->m_group, keep);
+    k_compact<<<grid_cols, blk, 0, st>>>(keep, h->k, h->kk, h->kk_pad, h->n_keep, h->m_group, h->c_in, h->kw,
+                                         h->indices, h->taps);
+    k_gather_values<<<grid_vals, blk, 0, st>>>(w_dense, h->indices, h->k, h->kk, h->kk_pad, h->tile_t, h->values,
+                                               h->wt);
+    count_launch(4);
+    NM_CUDA_TRY(cudaGetLastError());
+    NM_CUDA_TRY(cudaStreamSynchronize(st));  // the scratch is freed below
+done:
+    cudaFree(score);
+    cudaFree(keep);
+    return st_out;
+}
+
+nm_status_t build_from_compressed(const float* values, const uint16_t* indices, nm_weights* h, cudaStream_t st)
+{
+    nm_status_t st_out = NM_OK;
+    int bad = 0;
+    const dim3 blk(128);
+    const dim3 grid_idx((h->kk + 127) / 128, h->n_tiles);
+    const dim3 grid_vals((h->kk_pad + 127) / 128, h->c_out);
+    NM_CUDA_TRY(cudaMemcpyAsync(h->values, values, static_cast<size_t>(h->c_out) * h->kk * sizeof(float),
+                                cudaMemcpyDeviceToDevice, st));
+    NM_CUDA_TRY(cudaMemcpyAsync(h->indices, indices, static_cast<size_t>(h->n_tiles) * h->kk * sizeof(uint16_t),
+                                cudaMemcpyDeviceToDevice, st));
+    NM_CUDA_TRY(cudaMemsetAsync(h->taps, 0xFF, static_cast<size_t>(h->n_tiles) * h->kk_pad * sizeof(uint32_t), st));
+    NM_CUDA_TRY(cudaMemsetAsync(h->status + 3, 0, sizeof(int), st));
+    if (h->kk > 0) {
+        k_check_indices<<<grid_idx, blk, 0, st>>>(h->indices, h->kk, h->k, h->status + 3);
+        k_taps_from_indices<<<grid_idx, blk, 0, st>>>(h->indices, h->kk, h->kk_pad, h->c_in, h->kw, h->taps);
+        count_launch(2);
+    }
+    k_round_values<<<grid_vals, blk, 0, st>>>(h->values, h->kk, h->kk_pad, h->wt);
+    count_launch(1);
+    NM_CUDA_TRY(cudaGetLastError());
+    NM_CUDA_TRY(cudaMemcpyAsync(&bad, h->status + 3, sizeof(int), cudaMemcpyDeviceToHost, st));
+    NM_CUDA_TRY(cudaStreamSynchronize(st));
+    if (bad) st_out = fail(NM_ERR_INVALID_ARG, "nm_weights_import: an index row is not strictly ascending below K");
+done:
+    return st_out;
+}
+
+}  // namespace nmhost

@@ -1,0 +1,64 @@
+"""The C-ABI library loads and exports every symbol include/nm.h declares (no compute, no GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib_path():
+    from paper_2507_17301_b200 import build
+    return build.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "nm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(nm_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_three_calls():
+    names = _declared()
+    for must in ("nm_prune", "nm_conv2d", "nm_autotune"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(lib_path):
+    lib = ctypes.CDLL(lib_path)
+    for name in _declared():
+        assert hasattr(lib, name), f"{name} is declared in nm.h but not exported"
+
+
+def test_binding_names_match_header(lib_path):
+    from paper_2507_17301_b200 import nm
+    assert sorted(nm.EXPORTS) == _declared()
+    for name in nm.EXPORTS:
+        assert hasattr(nm, name) or hasattr(nm._lib, name)
+
+
+def test_argument_errors_without_gpu(lib_path):
+    from paper_2507_17301_b200 import nm
+    out = ctypes.c_void_p()
+    assert nm._lib.nm_prune(None, 8, 1, 1, 8, 2, 4, 8, None, ctypes.byref(out)) == nm.NM_ERR_INVALID_ARG
+    assert "NULL" in nm.nm_last_error()
+    fake = ctypes.c_void_p(16)
+    assert nm._lib.nm_prune(fake, 8, 1, 1, 8, 5, 4, 8, None, ctypes.byref(out)) == nm.NM_ERR_INVALID_ARG
+    assert nm._lib.nm_prune(fake, 8, 1, 1, 8, 0, 4, 8, None, ctypes.byref(out)) == nm.NM_ERR_INVALID_ARG
+    assert nm._lib.nm_prune(fake, 8, 3, 3, 8192, 2, 4, 8, None, ctypes.byref(out)) == nm.NM_ERR_UNSUPPORTED
+    assert nm._lib.nm_prune(fake, 8, 1, 1, 8, 2, 4, 512, None, ctypes.byref(out)) == nm.NM_ERR_UNSUPPORTED
+    assert nm._lib.nm_weights_dims(None, None, None, None, None, None) == nm.NM_ERR_INVALID_ARG
+    assert nm._lib.nm_weights_free(None) == nm.NM_OK
+    assert nm._status_string(nm.NM_ERR_TIMEOUT) == "NM_ERR_TIMEOUT"
+
+
+def test_product_path_does_not_touch_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2507_17301_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                for needle in ("import oracle", "from oracle", "nm_oracle", "oracle/"):
+                    assert needle not in text, f"{f} reaches for the CPU oracle ({needle})"

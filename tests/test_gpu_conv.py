@@ -1,0 +1,153 @@
+"""GPU convolution (nm_conv2d through the C ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_17301_b200 import inputs
+from paper_2507_17301_b200.inputs import ConvShape
+from parity import (assert_conv_close, assert_prune_bit_exact, errors, gpu_layer, oracle_layer, tensors_for)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nm():
+    from paper_2507_17301_b200 import nm as mod
+    return mod
+
+
+def _plans(nm, s):
+    """Every kernel variant that admits the shape, plus the library default."""
+    out = [None]
+    for variant in (1, 2):
+        p = nm.nm_plan_t()
+        p.variant = variant
+        out.append(p)
+    return out
+
+
+def _run(nm, s, integer=False, use_bias=True):
+    w, x, b = tensors_for(s, integer)
+    vr, ir, yr = oracle_layer(s, w, x, b, use_bias)
+    ran = 0
+    for plan in _plans(nm, s):
+        try:
+            _, v, i, y = gpu_layer(nm, s, w, x, b, use_bias, plan)
+        except nm.NmError as e:
+            if plan is not None and e.status == nm.NM_ERR_UNSUPPORTED:
+                continue  # this variant does not take the shape
+            raise
+        ran += 1
+        assert_prune_bit_exact(v, i, vr, ir)
+        if integer:
+            # every product and partial sum is exact in TF32 / fp32: results must be identical
+            assert np.array_equal(y, yr), f"integer case differs (variant {plan.variant if plan else 0})"
+        else:
+            assert_conv_close(y, yr)
+    assert ran >= 2  # the default and at least one explicit variant
+
+
+def test_tiny_config(nm):
+    _run(nm, inputs.config_tiny())
+
+
+def test_tiny_config_integer_exact(nm):
+    _run(nm, inputs.config_tiny(), integer=True)
+
+
+SMALL = [
+    ConvShape("s1_3x3_T8", 2, 9, 11, 16, 24, 3, 3, 1, 1, 1, 2, 4, 8),
+    ConvShape("ragged_pixels", 3, 13, 13, 32, 32, 3, 3, 1, 1, 1, 2, 4, 32),        # 507 pixels: 3 full tiles + tail
+    ConvShape("stride2", 2, 15, 15, 32, 64, 3, 3, 2, 1, 1, 2, 4, 32),
+    ConvShape("dilation2", 1, 12, 12, 16, 16, 3, 3, 1, 2, 2, 1, 4, 16),
+    ConvShape("one_by_one", 2, 7, 7, 64, 48, 1, 1, 1, 0, 1, 2, 4, 16),
+    ConvShape("one_by_one_s2", 2, 14, 14, 64, 32, 1, 1, 2, 0, 1, 1, 8, 32),
+    ConvShape("tail_tile", 1, 8, 8, 16, 40, 3, 3, 1, 1, 1, 2, 4, 16),               # c_out % T != 0
+    ConvShape("tail_group", 1, 8, 8, 6, 8, 3, 3, 1, 1, 1, 3, 4, 8),                 # K = 54, c_in % 4 != 0
+    ConvShape("t1_rowwise", 1, 6, 6, 16, 12, 3, 3, 1, 1, 1, 2, 4, 1),               # T = 1
+    ConvShape("odd_tile", 1, 6, 6, 16, 21, 1, 1, 1, 0, 1, 2, 4, 7),                 # T = 7
+    ConvShape("keep_all", 1, 10, 10, 8, 16, 3, 3, 1, 1, 1, 4, 4, 16),               # N = M: dense
+    ConvShape("stem_like", 1, 32, 32, 3, 64, 7, 7, 2, 3, 1, 1, 1, 64),              # 7x7, c_in = 3, dense
+    ConvShape("big_tile", 1, 12, 12, 64, 256, 3, 3, 1, 1, 1, 2, 8, 128),
+    ConvShape("tile256", 1, 12, 12, 32, 256, 1, 1, 1, 0, 1, 1, 4, 256),
+    ConvShape("no_pad_5x5", 1, 11, 11, 8, 8, 5, 5, 1, 0, 1, 2, 4, 8),
+    ConvShape("single_pixel", 1, 3, 3, 16, 16, 3, 3, 1, 0, 1, 2, 4, 16),            # one output pixel
+]
+
+
+@pytest.mark.parametrize("s", SMALL, ids=lambda s: s.name)
+def test_small_shapes(nm, s):
+    _run(nm, s)
+
+
+@pytest.mark.parametrize("s", SMALL[:8], ids=lambda s: s.name)
+def test_small_shapes_integer_exact(nm, s):
+    _run(nm, s, integer=True)
+
+
+def test_no_bias_no_relu(nm):
+    _run(nm, SMALL[0].with_(relu=False), use_bias=False)
+
+
+@pytest.mark.parametrize("s", inputs.config_resnet3x3(), ids=lambda s: s.name)
+def test_resnet3x3_full_layer(nm, s):
+    _run(nm, s)
+
+
+@pytest.mark.parametrize("s", [c.with_(batch=8) for c in inputs.config_bottleneck1x1()], ids=lambda s: s.name)
+def test_bottleneck1x1_batch8(nm, s):
+    _run(nm, s)
+
+
+def test_argument_errors(nm):
+    s = inputs.config_tiny()
+    w, x, b = tensors_for(s)
+    hnd = nm.nm_prune(w.cuda(), 2, 4, 8)
+    xd = x.cuda()
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_conv2d(hnd, xd, 3, 3, 0, 1, 1)              # stride 0
+    assert e.value.status == nm.NM_ERR_INVALID_ARG
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_conv2d(hnd, xd[:, :2, :2].contiguous(), 3, 3, 1, 0, 1)   # kernel larger than the image
+    assert e.value.status == nm.NM_ERR_INVALID_ARG
+    bad = torch.zeros(xd.numel() + 1, device="cuda")[1:].view_as(xd)   # 4-byte aligned only
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_conv2d(hnd, bad, 3, 3, 1, 1, 1)
+    assert e.value.status == nm.NM_ERR_INVALID_ARG
+    plan = nm.nm_plan_t()
+    plan.variant = 99
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_conv2d(hnd, xd, 3, 3, 1, 1, 1, plan=plan)
+    assert e.value.status == nm.NM_ERR_UNSUPPORTED
+    # the context is still usable afterwards
+    y = nm.nm_conv2d(hnd, xd, 3, 3, 1, 1, 1)
+    torch.cuda.synchronize()
+    assert torch.isfinite(y).all()
+
+
+def test_host_buffer_entry_point(nm):
+    s = inputs.config_tiny()
+    w, x, b = tensors_for(s)
+    _, _, yr = oracle_layer(s, w, x, b)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    xh, bh = x.pin_memory(), b.pin_memory()
+    yh = torch.empty(yr.shape, dtype=torch.float32).pin_memory()
+    xd, bd, yd = torch.empty_like(x, device="cuda"), torch.empty_like(b, device="cuda"), torch.empty(yr.shape, device="cuda")
+    nm.nm_conv2d_host(hnd, xh, xd, s.stride, s.pad, s.dil, bh, bd, s.relu, yh, yd)
+    torch.cuda.synchronize()
+    assert_conv_close(yh.numpy(), yr)
+
+
+def test_autotune_returns_a_working_plan(nm):
+    s = SMALL[1]
+    w, x, b = tensors_for(s)
+    _, _, yr = oracle_layer(s, w, x, b)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    plan, ms = nm.nm_autotune(hnd, x.cuda(), s.stride, s.pad, s.dil, b.cuda(), s.relu, kh=s.kh, kw=s.kw)
+    assert plan.variant >= 1 and ms > 0
+    y = nm.nm_conv2d(hnd, x.cuda(), s.kh, s.kw, s.stride, s.pad, s.dil, b.cuda(), s.relu, plan=plan)
+    torch.cuda.synchronize()
+    assert_conv_close(y.cpu().numpy(), yr)
+    tile, plan, ms = nm.nm_autotune_tile(w.cuda(), s.n_keep, s.m_group, [16, 32], x.cuda(), s.stride, s.pad, s.dil,
+                                         b.cuda(), s.relu)
+    assert tile in (16, 32) and ms > 0

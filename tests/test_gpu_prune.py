@@ -1,0 +1,82 @@
+"""GPU pruning (nm_prune through the C ABI) against the CPU oracle: bit-exact indices and values."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2507_17301_b200 import inputs
+from parity import assert_prune_bit_exact
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nm():
+    from paper_2507_17301_b200 import nm as mod
+    return mod
+
+
+def _check(nm, w, n, m, t):
+    hnd = nm.nm_prune(w.cuda(), n, m, t)
+    v, i = nm.nm_weights_export(hnd)
+    torch.cuda.synchronize()
+    vr, ir = oracle.prune(w.numpy(), n, m, t)
+    assert_prune_bit_exact(v.cpu().numpy(), i.cpu().numpy(), vr, ir)
+    assert (hnd.kk, hnd.n_tiles) == (vr.shape[1], ir.shape[0])
+    return hnd
+
+
+def test_tiny_config(nm):
+    s = inputs.config_tiny()
+    _check(nm, inputs.make_weights(s), s.n_keep, s.m_group, s.tile_t)
+
+
+@pytest.mark.parametrize("s", inputs.config_resnet3x3(), ids=lambda s: s.name)
+def test_resnet3x3_configs(nm, s):
+    _check(nm, inputs.make_weights(s), s.n_keep, s.m_group, s.tile_t)
+
+
+@pytest.mark.parametrize("s", inputs.config_bottleneck1x1(), ids=lambda s: s.name)
+def test_bottleneck_configs(nm, s):
+    _check(nm, inputs.make_weights(s), s.n_keep, s.m_group, s.tile_t)
+
+
+@pytest.mark.parametrize("n,m,t,c_out,shape", [
+    (3, 4, 5, 17, (5, 2, 5)),     # K = 50: tail group; tail tile
+    (1, 8, 1, 9, (1, 1, 72)),     # T = 1: row-wise N:M
+    (7, 16, 3, 10, (2, 5, 10)),
+    (4, 4, 8, 24, (3, 3, 7)),     # N = M keeps everything
+    (64, 128, 32, 64, (3, 3, 128)),   # adaptive-style large group
+    (2, 4, 256, 512, (1, 1, 64)),
+])
+def test_odd_shapes(nm, n, m, t, c_out, shape):
+    g = torch.Generator().manual_seed(n * 100 + m)
+    w = torch.randn((c_out,) + shape, generator=g)
+    _check(nm, w, n, m, t)
+
+
+def test_ties_resolve_like_the_oracle(nm):
+    g = torch.Generator().manual_seed(3)
+    w = torch.randint(-2, 3, (32, 3, 3, 16), generator=g).float()  # few distinct scores: many ties
+    _check(nm, w, 2, 4, 8)
+    _check(nm, w, 1, 8, 4)
+    _check(nm, torch.zeros(16, 1, 1, 32), 2, 4, 8)
+
+
+def test_import_round_trip_and_validation(nm):
+    s = inputs.config_tiny()
+    w = inputs.make_weights(s)
+    hnd = _check(nm, w, 2, 4, 8)
+    v, i = nm.nm_weights_export(hnd)
+    h2 = nm.nm_weights_import(v, i, 3, 3, 16, 2, 4, 8)
+    v2, i2 = nm.nm_weights_export(h2)
+    assert torch.equal(v, v2) and torch.equal(i.view(torch.int16), i2.view(torch.int16))
+    x = inputs.make_activations(s).cuda()
+    y1 = nm.nm_conv2d(hnd, x, 3, 3, 1, 1, 1)
+    y2 = nm.nm_conv2d(h2, x, 3, 3, 1, 1, 1)
+    assert torch.equal(y1, y2)
+    bad = i.clone().view(torch.int16)
+    bad[0, 1] = bad[0, 0]
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_weights_import(v, bad.view(torch.uint16), 3, 3, 16, 2, 4, 8)
+    assert e.value.status == nm.NM_ERR_INVALID_ARG

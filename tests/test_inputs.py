@@ -1,0 +1,32 @@
+"""The seeded input recipes are deterministic and have the stated shapes / sizes."""
+import torch
+
+from paper_2507_17301_b200 import inputs
+
+
+def test_seeded_draws_repeat():
+    s = inputs.config_tiny()
+    assert torch.equal(inputs.make_weights(s), inputs.make_weights(s))
+    assert torch.equal(inputs.make_activations(s), inputs.make_activations(s))
+    assert not torch.equal(inputs.make_weights(s, 1), inputs.make_weights(s, 0))
+    assert inputs.make_weights(s).shape == (32, 3, 3, 16)
+    assert inputs.make_activations(s).shape == (1, 14, 14, 16)
+    assert (s.k, s.kk, s.pixels, s.ho, s.wo) == (144, 72, 196, 14, 14)
+
+
+def test_kaiming_scale():
+    s = inputs.config_resnet3x3()[0]
+    w = inputs.make_weights(s)
+    assert abs(float(w.std()) - (2.0 / s.k) ** 0.5) < 0.02 * (2.0 / s.k) ** 0.5
+
+
+def test_resnet_stacks_have_the_published_conv_counts_and_flops():
+    r50 = inputs.resnet_conv_stack(50, 64, 2, 4)
+    assert len(r50) == 53
+    dense = sum(2 * s.pixels * s.c_out * s.k for s in r50) / 64
+    assert abs(dense / 1e9 - 8.17) < 0.1  # ~4.1 GMAC per image
+    r101 = inputs.resnet_conv_stack(101, 128, 1, 4)
+    assert len(r101) == 104
+    assert r50[0].kk == r50[0].k == 147  # stem keeps every column
+    # spatial sizes chain: last block works on 7x7
+    assert (r50[-1].ho, r50[-1].c_out) == (7, 2048)
