@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the column-wise N:M sparse-convolution hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload: every convolution of ResNet-50 at 224x224, batch 64 per GPU (53 layers; the 7x7 stem
+keeps all its columns, every other layer is pruned column-wise 2:4), seeded synthetic inputs
+(activations N(0,1), Kaiming-normal weights, bias N(0,1)); each layer runs on its own input
+tensor of the right shape.  One step = one pass over all 53 layers through the C ABI.
+
+Prints ONE JSON line: images/s over all GPUs (inputs resident in HBM), the same through the
+host-buffer entry point (`e2e`), a roofline object (algorithmic bytes per step / measured time
+against the measured HBM copy peak), the CPU checker timed on a bounded sample (`cpu_baseline`),
+clocks sampled during the timed region, and a per-layer table (time, useful TFLOP/s, fraction of
+max(kept FLOPs / TF32 peak, bytes / HBM peak)).  `--impl reference` times the CPU checker instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2507_17301_b200 import inputs  # noqa: E402
+
+METRIC = "resnet50_conv_stack_images_per_s"
+UNIT = "images/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "source": "fallback"}
+
+
+def algorithmic_bytes(s: inputs.ConvShape) -> int:
+    """Bytes one layer must move, each distinct byte once: input touched + output + compressed
+    weights + indices + bias.  A strided 1x1 conv touches only the pixels it samples."""
+    if s.kh == 1 and s.kw == 1 and s.stride > 1:
+        in_elems = s.pixels * s.c_in
+    else:
+        in_elems = s.batch * s.h * s.w * s.c_in
+    n_tiles = -(-s.c_out // s.tile_t)
+    return 4 * in_elems + 4 * s.pixels * s.c_out + 4 * s.c_out * s.kk + 2 * n_tiles * s.kk + 4 * s.c_out
+
+
+def useful_flops(s: inputs.ConvShape) -> int:
+    return 2 * s.pixels * s.c_out * s.kk
+
+
+def workload(batch: int):
+    return inputs.resnet_conv_stack(50, batch, 2, 4, tile_t=64)
+
+
+class ClockSampler:
+    """Polls nvidia-smi for SM clock and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [v for v in sm if v > 0.5 * (max(mx) if mx else 1)] or sm
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(value: float, world: int) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def measure_tf32_peak() -> float:
+    """Dense TF32 matmul throughput (library GEMM, 8192^3, best of 10): the tensor roof per layer."""
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        n = 8192
+        a = torch.randn(n, n, device="cuda")
+        b = torch.randn(n, n, device="cuda")
+        for _ in range(3):
+            a @ b
+        best = 1e9
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+            e0.record()
+            a @ b
+            e1.record()
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 2 * n ** 3 / (best * 1e-3) / 1e12
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+
+
+def run_reference(args):
+    """The CPU checker, as it stands, on a bounded sample: image 0 of every layer of the stack."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    layers = workload(1)
+    prepared = []
+    for li, s in enumerate(layers):
+        w = inputs.make_weights(s, li)
+        values, indices = oracle.prune(w.numpy(), s.n_keep, s.m_group, s.tile_t)
+        prepared.append((s, values, indices, inputs.make_activations(s, li, batch=1).numpy(), inputs.make_bias(s, li).numpy()))
+
+    def step():
+        for s, values, indices, x, b in prepared:
+            oracle.conv2d(values, indices, s.kh, s.kw, s.c_in, s.tile_t, x, (s.stride,) * 2, (s.pad,) * 2,
+                          (s.dil,) * 2, b, s.relu)
+
+    steps = max(1, min(args.steps, 5))
+    for _ in range(min(args.warmup, 1)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    value = 1.0 / dt
+    sample = "image 0 of each of the 53 layers per step (1 of 64 images)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "resnet50_conv_stack_b64_224_2of4", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(budget_s: float = 20.0):
+    import oracle
+    layers = workload(1)
+    t_total, done = 0.0, 0
+    t_begin = time.perf_counter()
+    for li, s in enumerate(layers):
+        w = inputs.make_weights(s, li)
+        values, indices = oracle.prune(w.numpy(), s.n_keep, s.m_group, s.tile_t)
+        x = inputs.make_activations(s, li, batch=1).numpy()
+        b = inputs.make_bias(s, li).numpy()
+        t0 = time.perf_counter()
+        oracle.conv2d(values, indices, s.kh, s.kw, s.c_in, s.tile_t, x, (s.stride,) * 2, (s.pad,) * 2, (s.dil,) * 2, b,
+                      s.relu)
+        t_total += time.perf_counter() - t0
+        done += 1
+        if time.perf_counter() - t_begin > budget_s * 3:
+            break
+    flops_done = sum(useful_flops(s) for s in layers[:done])
+    flops_all = sum(useful_flops(s) for s in layers)
+    est_image_s = t_total * flops_all / flops_done  # scaled by kept FLOPs if the budget cut the pass short
+    sample = (f"image 0 of the first {done} of 53 layers (1 of 64 images)"
+              + ("" if done == len(layers) else ", scaled to the stack by kept FLOPs"))
+    return {"value": 1.0 / est_image_s, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline, cuDNN and per-layer passes")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    world, rank, local = dist_setup(args.gpus)
+    from paper_2507_17301_b200 import build
+    if rank == 0:
+        build.build()
+    barrier(world)
+    from paper_2507_17301_b200 import nm  # fails loudly if the CUDA library is missing
+
+    pk = peaks()
+    layers = workload(args.batch)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    state = []
+    for li, s in enumerate(layers):
+        w = inputs.make_weights(s, li).to(dev)
+        hnd = nm.nm_prune(w, s.n_keep, s.m_group, s.tile_t)
+        del w
+        g = torch.Generator(device="cpu").manual_seed(1 + 1000 * li + 7919 * rank)
+        # activations ~ N(0,1): drawn on the host in slices to bound pinned/pageable staging
+        x = torch.empty((s.batch, s.h, s.w, s.c_in), dtype=torch.float32, device=dev)
+        for b0 in range(0, s.batch, 8):
+            x[b0:b0 + 8] = torch.randn((min(8, s.batch - b0), s.h, s.w, s.c_in), generator=g).to(dev)
+        bias = inputs.make_bias(s, li).to(dev)
+        y = torch.empty((s.batch, s.ho, s.wo, s.c_out), dtype=torch.float32, device=dev)
+        plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
+        state.append((s, hnd, x, bias, y, plan))
+
+    def step():
+        for s, hnd, x, bias, y, plan in state:
+            nm.nm_conv2d(hnd, x, s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=y, plan=plan)
+
+    for _ in range(args.warmup):
+        step()
+    barrier(world)
+    sampler = ClockSampler(local if world > 1 else 0)
+    if rank == 0:
+        sampler.start()
+    launches0 = nm.nm_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier(world)
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world)
+    launches = nm.nm_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    for s, hnd, *_ in state:
+        nm.nm_weights_check(hnd)
+    ms_step = ms_total / args.steps
+    value = world * args.batch / (ms_step * 1e-3)
+
+    bytes_step = sum(algorithmic_bytes(s) for s in layers)
+    flops_step = sum(useful_flops(s) for s in layers)
+    achieved_gbs = bytes_step / (ms_step * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
+        "data": "synthetic",
+        "config": {"workload": "resnet50_conv_stack_b64_224_2of4", "layers": len(layers), "batch_per_gpu": args.batch,
+                   "tile_t": 64, "cache": "inputs larger than L2 (5.4 GB touched per step, one buffer per layer)",
+                   "parallelism": f"replicas x{world}"},
+        "useful_tflops": flops_step / (ms_step * 1e-3) / 1e12,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved_gbs / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"],
+                     "kernel": "conv kernels of the whole stack (53 launches per step)"},
+    }
+
+    if rank == 0 and not args.no_extras and world == 1:
+        tf32_peak = measure_tf32_peak()
+        out["tf32_peak_tflops_measured"] = tf32_peak
+        # per-layer pass: events around each launch, other layers' traffic in between keeps it cold
+        reps = 5
+        per = [[] for _ in state]
+        for _ in range(reps):
+            evs = []
+            for s, hnd, x, bias, y, plan in state:
+                a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+                a.record()
+                nm.nm_conv2d(hnd, x, s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=y, plan=plan)
+                b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            for i, (a, b) in enumerate(evs):
+                per[i].append(a.elapsed_time(b))
+        table, t_roof_sum = [], 0.0
+        for (s, hnd, x, bias, y, plan), ts in zip(state, per):
+            ms = statistics.median(ts)
+            t_tc = useful_flops(s) / (tf32_peak * 1e12) * 1e3
+            t_hbm = algorithmic_bytes(s) / (pk["hbm_gbs"] * 1e9) * 1e3
+            t_roof = max(t_tc, t_hbm)
+            t_roof_sum += t_roof
+            table.append({"layer": s.name, "shape": f"{s.c_in}->{s.c_out} {s.kh}x{s.kw}/{s.stride} @{s.h}",
+                          "ms": round(ms, 4), "useful_tflops": round(useful_flops(s) / (ms * 1e-3) / 1e12, 2),
+                          "gbs": round(algorithmic_bytes(s) / (ms * 1e-3) / 1e9, 1),
+                          "bound": "tensor" if t_tc > t_hbm else "hbm", "roofline_frac": round(t_roof / ms, 3),
+                          "plan": plan.as_dict()})
+        out["stack_roofline_frac"] = t_roof_sum / ms_step
+        out["per_layer"] = table
+
+        # cuDNN dense convolution on the same shapes (context, unpruned weights, TF32 allowed)
+        try:
+            torch.backends.cudnn.allow_tf32 = True
+            torch.backends.cudnn.benchmark = True
+            dense = []
+            for li, (s, hnd, x, bias, y, plan) in enumerate(state):
+                w = inputs.make_weights(s, li).to(dev).permute(0, 3, 1, 2).contiguous(memory_format=torch.channels_last)
+                dense.append((s, x.permute(0, 3, 1, 2), w, bias))
+            def dense_step():
+                for s, xx, w, b in dense:
+                    torch.nn.functional.conv2d(xx, w, b, stride=s.stride, padding=s.pad, dilation=s.dil)
+            for _ in range(3):
+                dense_step()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+            a.record()
+            for _ in range(5):
+                dense_step()
+            b.record()
+            b.synchronize()
+            out["cudnn_dense_images_per_s"] = args.batch / (a.elapsed_time(b) / 5 * 1e-3)
+            del dense
+        except Exception as exc:  # context only
+            out["cudnn_dense_images_per_s"] = f"unavailable: {exc}"
+
+        # end to end through the host-buffer entry point: pinned host x / y per layer
+        host = []
+        h2d = d2h = 0
+        for s, hnd, x, bias, y, plan in state:
+            xh = torch.empty(x.shape, dtype=torch.float32).pin_memory()
+            xh.copy_(x)
+            yh = torch.empty(y.shape, dtype=torch.float32).pin_memory()
+            bh = bias.cpu().pin_memory()
+            host.append((xh, bh, yh))
+            h2d += xh.numel() * 4 + bh.numel() * 4
+            d2h += yh.numel() * 4
+        def e2e_step():
+            for (s, hnd, x, bias, y, plan), (xh, bh, yh) in zip(state, host):
+                nm.nm_conv2d_host(hnd, xh, x, s.stride, s.pad, s.dil, bh, bias, s.relu, yh, y, plan=plan)
+        e2e_step()
+        torch.cuda.synchronize()
+        n_e2e = max(1, min(args.steps, 3))
+        a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record()
+        b.synchronize()
+        out["e2e"] = {"value": args.batch / (a.elapsed_time(b) / n_e2e * 1e-3), "unit": UNIT,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
+                      "note": "every layer's input copied from pinned host memory and every output copied back"}
+        del host
+        out["cpu_baseline"] = cpu_baseline()
+
+    if rank == 0:
+        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+        with open(os.path.join(ROOT, "gpurun_out", "bench_last.json"), "w") as f:
+            json.dump(out, f, indent=1)
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

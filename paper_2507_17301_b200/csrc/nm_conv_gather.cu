@@ -187,11 +187,10 @@ nm_status_t launch_conv_gather(const ConvParams& p, cudaStream_t st)
     const size_t floor_bytes = (227 * 1024) / (max_ctas + 1) + 1;
     if (max_ctas < 16 && smem < floor_bytes) smem = floor_bytes;
 
-    static thread_local size_t configured = 0;
-    if (smem > 48 * 1024 && smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(k_conv_gather, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(k_conv_gather, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
         if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        configured = 227 * 1024;
     }
     const long long tiles_m = (p.pixels + BM - 1) / BM;
     if (tiles_m > 0x7FFFFFFFll) return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: too many output pixels");

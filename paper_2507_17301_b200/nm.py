@@ -181,7 +181,11 @@ def nm_conv2d(w: Weights, x: torch.Tensor, kh: int, kw: int, stride=1, pad=0, di
     xp = _dev_f32(x, "x")
     b, h, wd, _ = x.shape
     if y is None:
-        y = torch.empty(out_shape(x.shape, kh, kw, w.c_out, stride, pad, dil), dtype=torch.float32, device=x.device)
+        if min(stride) < 1 or min(dil) < 1:  # let the library report it
+            y = torch.empty(4, dtype=torch.float32, device=x.device)
+        else:
+            shape = out_shape(x.shape, kh, kw, w.c_out, stride, pad, dil)
+            y = torch.empty([max(d, 1) for d in shape], dtype=torch.float32, device=x.device)
     yp = _dev_f32(y, "y")
     bp = _dev_f32(bias, "bias") if bias is not None else None
     _check(_lib.nm_conv2d(w.handle, xp, b, h, wd, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], bp,
