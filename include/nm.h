@@ -95,6 +95,30 @@ typedef struct {
 nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep,
                      int m_group, int tile_t, void* cuda_stream, nm_weights_t** out);
 
+/*
+ * nm_prune for callers that cannot allocate device memory (the paper has no counterpart; this is a
+ * deployment aid).  Meant for a plug-in living inside a process whose GPU memory is entirely
+ * managed by someone else's pool, where cudaMalloc fails or breaks the host's accounting, and for
+ * latency-critical loops that cannot afford the device-wide synchronisation cudaMalloc / cudaFree
+ * imply.  It performs the same pruning as nm_prune and produces the same canonical result, but
+ *   - writes it straight into caller memory: values  device fp32  [c_out][kk],
+ *                                            indices device uint16 [ceil(c_out/tile_t)][kk],
+ *     kk = N*(K / M) + min(N, K % M) (no handle is created; feed the pair to nm_weights_import
+ *     when a handle is wanted and allocation is possible);
+ *   - takes its scratch (fp64 scores and keep flags) from a fixed array compiled into the library,
+ *     resident on every GPU that loads it (about 4.5 MiB) until the process ends;
+ *   - calls no cudaMalloc, cudaFree or any other allocating routine.
+ * Limit: ceil(c_out / tile_t) * K <= NM_NOALLOC_MAX_CELLS and c_out <= 65535; beyond that it returns
+ * NM_ERR_UNSUPPORTED and does nothing.  All calls share the one scratch array: calls whose kernels
+ * could overlap on the GPU (other streams or threads) race, so issue them one after another on one
+ * stream.  The first call on a given device looks up the array's device address (once per device,
+ * cached); make that first call outside any stream capture.  Asynchronous on `cuda_stream`.
+ */
+#define NM_NOALLOC_MAX_CELLS (1 << 19)
+nm_status_t nm_prune_noalloc(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep,
+                             int m_group, int tile_t, float* values, uint16_t* indices,
+                             void* cuda_stream);
+
 /* Dimensions of a handle; any output pointer may be NULL. */
 nm_status_t nm_weights_dims(const nm_weights_t* w, int* c_out, int* k, int* kk, int* n_tiles,
                             int* tile_t);

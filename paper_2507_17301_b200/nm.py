@@ -48,6 +48,7 @@ def _load():
     ip = ctypes.POINTER(ctypes.c_int)
     pp = ctypes.POINTER(nm_plan_t)
     lib.nm_prune.argtypes = [vp, i, i, i, i, i, i, i, vp, ctypes.POINTER(vp)]
+    lib.nm_prune_noalloc.argtypes = [vp, i, i, i, i, i, i, i, vp, vp, vp]
     lib.nm_weights_dims.argtypes = [vp, ip, ip, ip, ip, ip]
     lib.nm_weights_export.argtypes = [vp, vp, vp, vp]
     lib.nm_weights_import.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, ctypes.POINTER(vp)]
@@ -58,7 +59,7 @@ def _load():
     lib.nm_conv2d_host.argtypes = [vp, vp, vp] + conv_geom + [vp, vp, i, vp, vp, pp, vp]
     lib.nm_autotune.argtypes = [vp, vp] + conv_geom + [vp, i, vp, vp, pp, fp]
     lib.nm_autotune_tile.argtypes = [vp, i, i, i, i, i, i, ip, i, vp] + conv_geom + [vp, i, vp, vp, ip, pp, fp]
-    for name in ("nm_prune", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+    for name in ("nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
                  "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile"):
         getattr(lib, name).restype = ctypes.c_int
     lib.nm_status_string.argtypes = [ctypes.c_int]
@@ -72,7 +73,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_prune", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -142,6 +143,27 @@ def nm_prune(w_dense: torch.Tensor, n_keep: int, m_group: int, tile_t: int) -> W
     out = ctypes.c_void_p()
     _check(_lib.nm_prune(ptr, c_out, kh, kw, c_in, n_keep, m_group, tile_t, _stream(), ctypes.byref(out)))
     return Weights(out.value)
+
+
+NM_NOALLOC_MAX_CELLS = 1 << 19
+
+
+def nm_prune_noalloc(w_dense: torch.Tensor, n_keep: int, m_group: int, tile_t: int, values: torch.Tensor,
+                     indices: torch.Tensor) -> None:
+    """Pruning for callers that must not allocate on the device (a plug-in inside a server that owns
+    all GPU memory, a loop that cannot afford cudaMalloc's synchronisation): the caller passes the
+    output tensors ``values [c_out, kk]`` fp32 and ``indices [n_tiles, kk]`` uint16, the library uses
+    its built-in scratch array and allocates nothing.  Problems with more than
+    ``NM_NOALLOC_MAX_CELLS`` (tile, column) cells are refused; calls must not overlap on the GPU."""
+    ptr = _dev_f32(w_dense, "w_dense")
+    if w_dense.dim() != 4:
+        raise TypeError("w_dense must be [c_out, kh, kw, c_in]")
+    c_out, kh, kw, c_in = w_dense.shape
+    vptr = _dev_f32(values, "values")
+    if not (indices.is_cuda and indices.dtype == torch.uint16 and indices.is_contiguous()):
+        raise TypeError("indices must be a contiguous uint16 CUDA tensor")
+    _check(_lib.nm_prune_noalloc(ptr, c_out, kh, kw, c_in, n_keep, m_group, tile_t, vptr, indices.data_ptr(),
+                                 _stream()))
 
 
 def nm_weights_export(w: Weights):
