@@ -79,7 +79,7 @@ typedef struct {
  * Rows of the [c_out, K] filter matrix are cut into tiles of `tile_t` output channels.  Inside a
  * tile a column (its tile_t weights) is one unit scored by its L1 norm; in every group of
  * `m_group` consecutive columns the `n_keep` highest-scoring units are RETAINED (N counts kept
- * columns: "N = (1 - sparsity) * M") and all rows of the tile share that kept set.
+ * columns, N = (1 - sparsity) * M) and all rows of the tile share that kept set.
  * Deterministic rules where the paper is silent: scores are fp64 sums over the tile's rows in
  * ascending row order; of two equal scores the lower column is kept; a tail group of m' < M
  * columns keeps min(N, m'); a tail tile (c_out % tile_t rows) scores over the rows it has.
@@ -124,8 +124,8 @@ nm_status_t nm_weights_dims(const nm_weights_t* w, int* c_out, int* k, int* kk, 
                             int* tile_t);
 
 /*
- * Copies the canonical compressed form (Sec. 2.1: "a compressed weight format and an index
- * array"; Algorithm 1 inputs W[T, N] and Idx[N]) to caller memory on `cuda_stream`:
+ * Copies the canonical compressed form (the compacted weights plus index array of Sec. 2.1,
+ * i.e. Algorithm 1's inputs W[T, N] and Idx[N]) to caller memory on `cuda_stream`:
  *   values   device, fp32 [c_out][kk]: values[o][j] = w[o][indices[o / tile_t][j]], bit-exact
  *   indices  device, uint16 [n_tiles][kk]: absolute column positions k, ascending
  * Either pointer may be NULL to skip it.

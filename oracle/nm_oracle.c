@@ -12,7 +12,7 @@
  *   - Rows are cut into tiles of T output channels; inside a tile one column (its
  *     T weights) is the pruning unit, scored by its L1 norm (Sec. 3.1).
  *   - In every group of M consecutive columns N units are RETAINED (Sec. 2.1,
- *     Sec. 3.1 "N = (1 - sparsity) * M", Algorithm 1 input "N").
+ *     Sec. 3.1: N = (1 - sparsity) * M; Algorithm 1 takes N as the retained count).
  *   - Compressed form: values W[T, kept] per tile plus the index array Idx[kept]
  *     holding the surviving column positions (Sec. 2.1, Algorithm 1 inputs).
  *   - The product is the plain matrix product on the retained columns
