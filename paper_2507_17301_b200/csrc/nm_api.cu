@@ -31,6 +31,8 @@ void free_handle_memory(nm_weights* h)
     cudaFree(h->wt);
     cudaFree(h->taps);
     cudaFree(h->status);
+    cudaFree(h->wt2);
+    cudaFree(h->rel2);
     h->magic = 0;
     delete h;
 }
@@ -112,6 +114,10 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     p->kk = w->kk; p->kk_pad = w->kk_pad; p->tile_t = w->tile_t; p->n_tiles = w->n_tiles; p->relu = relu ? 1 : 0;
     p->n_keep = w->n_keep; p->m_group = w->m_group;
     p->pixels = pixels;
+    p->k = w->k;
+    p->wt2 = w->v2_ok ? w->wt2 : nullptr;
+    p->rel2 = w->v2_ok ? w->rel2 : nullptr;
+    p->v2_kc = w->v2_kc; p->v2_s = w->v2_s; p->v2_chunks = w->v2_chunks;
     return NM_OK;
 }
 
@@ -120,18 +126,29 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
     const int variant = plan ? plan->variant : 0;
     switch (variant) {
         case 0:
+            if (nmhost::slab_plan_ok(p, nullptr)) return nmhost::launch_conv_slab(p, nullptr, st);
+            return nmhost::launch_conv_gather(p, st);
         case 1:
             return nmhost::launch_conv_gather(p, st);
+        case 2:
+            return nmhost::launch_conv_slab(p, plan, st);
         default:
             return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
     }
 }
 
 // Candidate plans for a layer, most promising first.
-std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams& /*p*/)
+std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams& p)
 {
     std::vector<nm_plan_t> out;
     nm_plan_t a;
+    std::memset(&a, 0, sizeof(a));
+    for (int bn : {0, p.tile_t}) {          // default (as many tiles as fit) and one tile per CTA
+        for (int stages : {2, 3}) {
+            a.variant = 2; a.bn = bn; a.stages = stages;
+            if (nmhost::slab_plan_ok(p, &a)) out.push_back(a);
+        }
+    }
     std::memset(&a, 0, sizeof(a));
     a.variant = 1;
     out.push_back(a);
@@ -162,6 +179,7 @@ nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, 
     nm_status_t s = make_handle("nm_prune", c_out, kh, kw, c_in, n_keep, m_group, tile_t, &h);
     if (s != NM_OK) return s;
     s = nmhost::prune_on_device(w_dense, h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         return s;
@@ -178,6 +196,7 @@ nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int 
     nm_status_t s = make_handle("nm_weights_import", c_out, kh, kw, c_in, n_keep, m_group, tile_t, &h);
     if (s != NM_OK) return s;
     s = nmhost::build_from_compressed(values, indices, h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         *out = nullptr;

@@ -21,6 +21,12 @@ struct nm_weights {
     float* wt;           // [c_out][kk_pad] retained weights rounded to TF32 (nearest), zero padded
     uint32_t* taps;      // [n_tiles][kk_pad] kh << 24 | kw << 16 | c per retained column, NM_TAP_PAD in the padding
     int* status;         // device int[4]: [0] error code, [1] where, [2] block, [3] spare
+    // Slab layout (variant 2); v2_ok = 0 when the N:M pattern does not fit it.
+    // The reduction axis is cut into chunks of v2_g whole groups: v2_s = g * M source columns, of
+    // which every tile keeps v2_kc = g * N (a multiple of 8, at most 32).
+    int v2_ok, v2_g, v2_kc, v2_s, v2_chunks;
+    float* wt2;          // [c_out][v2_chunks * 32] TF32 weights, chunk-major, first v2_kc of each 32 used
+    uint8_t* rel2;       // [n_tiles][v2_chunks * 32] source column of each kept column, relative to its chunk
 };
 
 // Geometry handed to the convolution kernels.
@@ -37,6 +43,11 @@ struct ConvParams {
     int kk, kk_pad, tile_t, n_tiles, relu;
     int n_keep, m_group;
     long long pixels;  // batch * ho * wo
+    int k;
+    // slab layout (variant 2)
+    const float* wt2;
+    const uint8_t* rel2;
+    int v2_kc, v2_s, v2_chunks;
 };
 
 namespace nmhost {
@@ -48,6 +59,12 @@ void count_launch(int n = 1);
 nm_status_t prune_on_device(const float* w_dense, nm_weights* h, cudaStream_t st);
 nm_status_t build_from_compressed(const float* values, const uint16_t* indices, nm_weights* h, cudaStream_t st);
 
+nm_status_t build_slab_layout(nm_weights* h, cudaStream_t st);
+
 // nm_conv_gather.cu — variant 1
 nm_status_t launch_conv_gather(const ConvParams& p, cudaStream_t st);
+
+// nm_conv_slab.cu — variant 2
+bool slab_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_slab(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 }  // namespace nmhost

@@ -102,6 +102,24 @@ __global__ void k_round_values(const float* __restrict__ values, int kk, int kk_
     wt[static_cast<size_t>(o) * kk_pad + j] = nmk::to_tf32(v);
 }
 
+// Slab layout: kept column j of a tile lies in chunk k_j / S at position j - chunk * KC (every
+// group before the last is full, so a chunk of G groups holds exactly KC = G * N kept columns).
+__global__ void k_build_slab(const float* __restrict__ values, const uint16_t* __restrict__ indices, int kk,
+                             int tile_t, int s_cols, int kc, int chunks, float* __restrict__ wt2,
+                             uint8_t* __restrict__ rel2)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int o = blockIdx.y;
+    if (j >= kk) return;
+    const int r = o / tile_t;
+    const int col = indices[static_cast<size_t>(r) * kk + j];
+    const int chunk = col / s_cols;
+    const int jj = j - chunk * kc;
+    const size_t pitch = static_cast<size_t>(chunks) * 32;
+    wt2[static_cast<size_t>(o) * pitch + chunk * 32 + jj] = nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
+    if (o == r * tile_t) rel2[static_cast<size_t>(r) * pitch + chunk * 32 + jj] = static_cast<uint8_t>(col - chunk * s_cols);
+}
+
 // Import path: every index row must be strictly ascending and below k.
 __global__ void k_check_indices(const uint16_t* __restrict__ indices, int kk, int k, int* __restrict__ bad)
 {
@@ -154,6 +172,38 @@ done:
     cudaFree(score);
     cudaFree(keep);
     return st_out;
+}
+
+nm_status_t build_slab_layout(nm_weights* h, cudaStream_t st)
+{
+    h->v2_ok = 0;
+    // keep-all is the 1:1 pattern; otherwise the chunk is the largest whole number of groups
+    // whose kept columns number a multiple of 8 up to 32 and whose source columns number <= 64
+    const int n = h->n_keep == h->m_group ? 1 : h->n_keep;
+    const int m = h->n_keep == h->m_group ? 1 : h->m_group;
+    int g = 0;
+    for (int cand = 32 / n; cand >= 1; --cand)
+        if ((cand * n) % 8 == 0 && cand * m <= 64) { g = cand; break; }
+    if (g == 0 || h->kk == 0) return NM_OK;
+    h->v2_g = g; h->v2_kc = g * n; h->v2_s = g * m;
+    h->v2_chunks = (h->k + h->v2_s - 1) / h->v2_s;
+    const size_t pitch = static_cast<size_t>(h->v2_chunks) * 32;
+    if (cudaMalloc(&h->wt2, static_cast<size_t>(h->c_out) * pitch * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&h->rel2, static_cast<size_t>(h->n_tiles) * pitch) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return fail(NM_ERR_ALLOC, "cannot allocate the slab-layout weights");
+    }
+    cudaError_t e = cudaMemsetAsync(h->wt2, 0, static_cast<size_t>(h->c_out) * pitch * sizeof(float), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->rel2, 0, static_cast<size_t>(h->n_tiles) * pitch, st);
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "slab layout memset: %s", cudaGetErrorString(e));
+    const dim3 grid((h->kk + 127) / 128, h->c_out);
+    k_build_slab<<<grid, 128, 0, st>>>(h->values, h->indices, h->kk, h->tile_t, h->v2_s, h->v2_kc, h->v2_chunks,
+                                       h->wt2, h->rel2);
+    count_launch(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "slab layout kernel: %s", cudaGetErrorString(e));
+    h->v2_ok = 1;
+    return NM_OK;
 }
 
 nm_status_t build_from_compressed(const float* values, const uint16_t* indices, nm_weights* h, cudaStream_t st)
