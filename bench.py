@@ -243,6 +243,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline, cuDNN and per-layer passes")
+    ap.add_argument("--layer", default=None, help="run only the layers whose name contains this text (profiling aid)")
+    ap.add_argument("--variant", type=int, default=None, help="force a kernel variant instead of auto-tuning")
+    ap.add_argument("--bn", type=int, default=0, help="with --variant: output channels per CTA")
+    ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -258,6 +262,9 @@ def main():
 
     pk = peaks()
     layers = workload(args.batch)
+    if args.layer:
+        layers = [s for s in layers if args.layer in s.name]
+        assert layers, f"no layer matches {args.layer!r}"
     dev = torch.device("cuda", local if world > 1 else 0)
     state = []
     for li, s in enumerate(layers):
@@ -271,7 +278,11 @@ def main():
             x[b0:b0 + 8] = torch.randn((min(8, s.batch - b0), s.h, s.w, s.c_in), generator=g).to(dev)
         bias = inputs.make_bias(s, li).to(dev)
         y = torch.empty((s.batch, s.ho, s.wo, s.c_out), dtype=torch.float32, device=dev)
-        plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
+        if args.variant is None:
+            plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
+        else:
+            plan = nm.nm_plan_t()
+            plan.variant, plan.bn, plan.stages = args.variant, args.bn, args.stages
         state.append((s, hnd, x, bias, y, plan))
 
     def step():
@@ -307,7 +318,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
         "data": "synthetic",
-        "config": {"workload": "resnet50_conv_stack_b64_224_2of4", "layers": len(layers), "batch_per_gpu": args.batch,
+        "config": {"workload": "resnet50_conv_stack_b64_224_2of4" + (f" [only {args.layer}]" if args.layer else ""),
+                   "layers": len(layers), "batch_per_gpu": args.batch,
                    "tile_t": 64, "cache": "inputs larger than L2 (5.4 GB touched per step, one buffer per layer)",
                    "parallelism": f"replicas x{world}"},
         "useful_tflops": flops_step / (ms_step * 1e-3) / 1e12,
