@@ -1,24 +1,30 @@
 // Variant 2: slab kernel — warp-specialised sparse implicit GEMM with the gathered operand in
 // tensor memory.
 //
-// One CTA owns 128 output pixels and up to NM_SLAB_MAX_TILES pruning tiles (<= 128 output
-// channels); two CTAs fit on an SM, so one CTA's epilogue overlaps the other's main loop.
-// The reduction axis is cut into chunks of G whole N:M groups (S = G*M source columns, of which
-// every tile keeps KC = G*N).  Per chunk:
-//   producers (4 warps)   cp.async the DENSE activation slab [128 pixels x S columns] once
-//                         (zero-filled outside the image; row pitch S+1 words so that a column can
-//                         be read by 32 pixels without bank conflicts) and the weight chunk
-//                         [channels x KC] in the 128-byte-swizzled K-major layout;
-//   compactors (4 warps)  thread = pixel; for each tile pick its KC kept columns out of the slab
-//                         by index (warp-uniform offsets), round to TF32 and write them to a TMEM
-//                         operand buffer with tcgen05.st  -> this is the fused im2col + packing
-//                         of Sec. 3.2 restricted to the surviving columns, with TMEM in the role
-//                         of the packed strip;
-//   MMA issuer (1 thread) D[128 x T] += A[tmem] * W_chunk[smem]^T, KC/8 tcgen05.mma per tile:
-//                         Algorithm 1's T accumulators are T TMEM columns.
+// One CTA owns 128 output pixels and as many pruning tiles as fit 128 accumulator columns; two
+// CTAs fit on an SM, so one CTA's epilogue overlaps the other's main loop.  The reduction axis
+// is cut into chunks of G whole N:M groups (S = G*M source columns, of which every tile keeps
+// KC = G*N).  Per chunk:
+//   producer      brings the DENSE activation slab [128 pixels x S columns] into shared memory
+//                 once, as 32-column sub-tiles in the 128-byte-swizzled layout, plus the weight
+//                 chunk [channels x KC] (same layout, K-major).  Fast path: one thread issues
+//                 TMA loads — im2col mode for the activations (the hardware walks the 128 output
+//                 pixels, applies stride / dilation / the tap offset and zero-fills the padding),
+//                 tiled mode for the weights.  General path (c_in % 32 != 0, tile_t % 8 != 0 or a
+//                 tensor under 128 KiB): four warps of 4-byte cp.async with the same layout.
+//   compactors    (4 warps, thread = pixel = TMEM lane) pick each tile's KC kept columns out of
+//                 the slab by index (warp-uniform offsets), round to TF32 and write them to a
+//                 TMEM operand buffer with tcgen05.st: the fused im2col + packing of Sec. 3.2
+//                 restricted to the surviving columns, TMEM standing in for the packed strip;
+//   MMA issuer    (1 thread) D[128 x T] += A[tmem] * W_chunk[smem]^T, KC/8 tcgen05.mma per tile:
+//                 Algorithm 1's T accumulator registers are T TMEM columns.
 // Epilogue (the compactor warps): TMEM -> registers, + bias, ReLU, NHWC store.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports through the
 // status word and drains to the common exit where TMEM is released.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "nm_internal.h"
 #include "nm_ptx.cuh"
 
@@ -31,20 +37,35 @@ constexpr int MAX_BN_COLS = 128;   // accumulator columns per CTA
 constexpr int NA = 4;              // TMEM operand buffers of 32 columns
 constexpr int TMEM_COLS = 256;     // 128 accumulator + 4 x 32 operand columns
 constexpr int NSTAGE_MAX = 4;
+constexpr int SUB_BYTES = BM * 128;  // one 32-column slab sub-tile
 
 struct SlabCfg {
     int g_tiles;      // pruning tiles per CTA
     int umma_n;       // accumulator columns per tile (tile_t rounded up to 16)
     int n_slices;     // CTAs along the channel axis
     int stages;
-    int slab_pitch;   // words per slab row (S + 1, odd)
-    int slab_bytes, b_bytes, stage_bytes;
+    int segs;         // 32-column sub-tiles per slab chunk
+    int b_rows;       // weight rows staged per chunk
+    int b_tile_rows;  // row distance between two tiles' weights in shared memory
+    int b_bytes, stage_bytes;
+    int use_tma;
 };
 
 __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
 
-template <int KC>
-__global__ void __launch_bounds__(288, 2) k_conv_slab(const ConvParams p, const SlabCfg cfg)
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const void* tmap, uint32_t bar, int c, int w, int h,
+                                                   int n, uint16_t off_w, uint16_t off_h)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cta.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+
+template <int KC, bool TMA>
+__global__ void __launch_bounds__(288, 2)
+k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUtensorMap tm_x,
+            const __grid_constant__ CUtensorMap tm_w)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[NSTAGE_MAX], s_free[NSTAGE_MAX], s_aready[NA], s_afree[NA], s_dready;
@@ -60,25 +81,29 @@ __global__ void __launch_bounds__(288, 2) k_conv_slab(const ConvParams p, const 
     const int g_here = min(cfg.g_tiles, p.n_tiles - tile0);
     const int S = p.v2_s, n_chunks = p.v2_chunks, NS = cfg.stages;
 
-    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;  // stage: [B tile (1024-aligned)][slab]
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;  // stage: [weight tile][slab sub-tiles]
     volatile int* abort_flag = &s_abort;
 
     // ---- set-up ----------------------------------------------------------------------------------
     if (warp == 8) tmem_alloc(smem_u32(&s_tmem), TMEM_COLS);
     if (tid == 0) {
         for (int i = 0; i < NSTAGE_MAX; ++i) {
-            mbar_init(smem_u32(&s_full[i]), 128);       // producer threads
-            mbar_init(smem_u32(&s_free[i]), 128 + 1);   // compactor threads + MMA commit
+            mbar_init(smem_u32(&s_full[i]), TMA ? 1 : 128);  // TMA issuer, or the producer threads
+            mbar_init(smem_u32(&s_free[i]), 128 + 1);        // compactor threads + MMA commit
         }
         for (int i = 0; i < NA; ++i) {
-            mbar_init(smem_u32(&s_aready[i]), 128);     // compactor threads
-            mbar_init(smem_u32(&s_afree[i]), 1);        // MMA commit
+            mbar_init(smem_u32(&s_aready[i]), 128);          // compactor threads
+            mbar_init(smem_u32(&s_afree[i]), 1);             // MMA commit
         }
         mbar_init(smem_u32(&s_dready), 1);
         mbar_fence_init();
         s_abort = 0;
+        if (TMA) {
+            tma_prefetch_desc(&tm_x);
+            tma_prefetch_desc(&tm_w);
+        }
     }
-    if (tid < BM) {
+    if (!TMA && tid < BM) {
         const long long pix = pix0 + tid;
         int off = 0;
         unsigned long long mask = 0;
@@ -103,75 +128,102 @@ __global__ void __launch_bounds__(288, 2) k_conv_slab(const ConvParams p, const 
     const uint32_t tmem = s_tmem;
 
     if (warp >= 4 && warp < 8) {
-        // =========================== producers ===========================
-        const int pw = warp - 4, ptid = tid - 128;
-        const int segs = (S + 31) / 32;
-        const int b_rows = cfg.g_tiles * cfg.umma_n;
-        constexpr int QPR = KC / 4;  // 16-byte pieces per weight row
-        const size_t wpitch = static_cast<size_t>(n_chunks) * 32;
-        for (int c = 0; c < n_chunks; ++c) {
-            const int s = c % NS;
-            if (c >= NS) {
-                if (!mbar_wait(smem_u32(&s_free[s]), ((c / NS) - 1) & 1)) { *abort_flag = 2; }
+        if (TMA) {
+            // =========================== TMA producer (one thread) ===========================
+            if (tid == 128) {
+                const int hw = p.ho * p.wo;
+                const int n0 = static_cast<int>(pix0 / hw);
+                const int rem = static_cast<int>(pix0 - static_cast<long long>(n0) * hw);
+                const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
+                const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
+                const uint32_t b_box_bytes = static_cast<uint32_t>(cfg.b_rows) * 128u;
+                for (int c = 0; c < n_chunks; ++c) {
+                    const int s = c % NS;
+                    if (c >= NS && !mbar_wait(smem_u32(&s_free[s]), ((c / NS) - 1) & 1)) *abort_flag = 2;
+                    if (aborted(abort_flag)) break;
+                    const uint32_t b_smem = ring + s * cfg.stage_bytes;
+                    const uint32_t slab = b_smem + cfg.b_bytes;
+                    const uint32_t bar = smem_u32(&s_full[s]);
+                    int live = 0;
+                    for (int seg = 0; seg < cfg.segs; ++seg) live += (c * S + seg * 32 < p.k) ? 1 : 0;
+                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(live) * SUB_BYTES + b_box_bytes);
+                    for (int seg = 0; seg < cfg.segs; ++seg) {
+                        const int k0 = c * S + seg * 32;
+                        if (k0 >= p.k) break;
+                        const int tap = k0 / p.c_in, cc = k0 - tap * p.c_in;
+                        tma_load_im2col_4d(slab + seg * SUB_BYTES, &tm_x, bar, cc, w0, h0, n0,
+                                           static_cast<uint16_t>((tap % p.kw) * p.dil_w),
+                                           static_cast<uint16_t>((tap / p.kw) * p.dil_h));
+                    }
+                    tma_load_2d(b_smem, &tm_w, bar, c * 32, tile0 * p.tile_t);
+                }
             }
-            if (aborted(abort_flag)) break;
-            const uint32_t b_smem = ring + s * cfg.stage_bytes;
-            const uint32_t slab = b_smem + cfg.b_bytes;
-            // activation slab: lane = source column, this warp's 32 pixels one after another
-            for (int seg = 0; seg < segs; ++seg) {
-                const int colc = seg * 32 + lane;            // column inside the chunk
-                const int k = c * S + colc;                  // flattened (kh, kw, c) column
-                const bool col_ok = colc < S && k < p.k;
-                const int tap = col_ok ? k / p.c_in : 0;
-                const int cc = col_ok ? k - tap * p.c_in : 0;
-                const int delta = ((tap / p.kw) * p.dil_h * p.w + (tap % p.kw) * p.dil_w) * p.c_in + cc;
-                const uint32_t dst0 = slab + static_cast<uint32_t>(colc) * 4u;
-                if (colc < S) {
+        } else {
+            // =========================== cp.async producers (4 warps) ===========================
+            const int pw = warp - 4, ptid = tid - 128;
+            constexpr int QPR = KC / 4;  // 16-byte pieces per weight row
+            const size_t wpitch = static_cast<size_t>(n_chunks) * 32;
+            for (int c = 0; c < n_chunks; ++c) {
+                const int s = c % NS;
+                if (c >= NS && !mbar_wait(smem_u32(&s_free[s]), ((c / NS) - 1) & 1)) *abort_flag = 2;
+                if (aborted(abort_flag)) break;
+                const uint32_t b_smem = ring + s * cfg.stage_bytes;
+                const uint32_t slab = b_smem + cfg.b_bytes;
+                // activation slab: lane = source column, this warp's 32 pixels one after another
+                for (int seg = 0; seg < cfg.segs; ++seg) {
+                    const int colc = seg * 32 + lane;            // column inside the chunk
+                    const int k = c * S + colc;                  // flattened (kh, kw, c) column
+                    const bool col_ok = colc < S && k < p.k;
+                    const int tap = col_ok ? k / p.c_in : 0;
+                    const int cc = col_ok ? k - tap * p.c_in : 0;
+                    const int delta = ((tap / p.kw) * p.dil_h * p.w + (tap % p.kw) * p.dil_w) * p.c_in + cc;
+                    const uint32_t dst0 = slab + seg * SUB_BYTES + ((lane & 3) << 2);
 #pragma unroll 4
                     for (int i = 0; i < 32; ++i) {
                         const int row = pw * 32 + i;
                         const bool ok = col_ok && ((s_rowmask[row] >> tap) & 1ull);
                         const float* src = ok ? p.x + (s_rowoff[row] + delta) : p.x;
-                        cp_async4(dst0 + static_cast<uint32_t>(row * cfg.slab_pitch) * 4u, src, ok ? 4u : 0u);
+                        cp_async4(dst0 + row * 128 + (((lane >> 2) ^ (row & 7)) << 4), src, ok ? 4u : 0u);
                     }
                 }
+                // weight chunk: rows = the CTA's channels (tile-major, umma_n rows per tile)
+                for (int piece = ptid; piece < cfg.b_rows * QPR; piece += 128) {
+                    const int row = piece / QPR, q = piece - row * QPR;
+                    const int t = row / cfg.umma_n, rr = row - t * cfg.umma_n;
+                    const int o = (tile0 + t) * p.tile_t + rr;
+                    const bool ok = t < g_here && rr < p.tile_t && o < p.c_out;
+                    const float* src = ok ? p.wt2 + static_cast<size_t>(o) * wpitch + c * 32 + q * 4 : p.wt2;
+                    cp_async16(b_smem + row * 128 + ((q ^ (row & 7)) << 4), src, ok ? 16u : 0u);
+                }
+                cp_async_commit();
+                // signal the previous chunk once its copies have landed (one group stays in flight)
+                if (c > 0) {
+                    cp_async_wait<1>();
+                    fence_proxy_async();
+                    mbar_arrive(smem_u32(&s_full[(c - 1) % NS]));
+                }
             }
-            // weight chunk: rows = the CTA's channels (tile-major, umma_n rows per tile)
-            for (int piece = ptid; piece < b_rows * QPR; piece += 128) {
-                const int row = piece / QPR, q = piece - row * QPR;
-                const int t = row / cfg.umma_n, rr = row - t * cfg.umma_n;
-                const int o = (tile0 + t) * p.tile_t + rr;
-                const bool ok = t < g_here && rr < p.tile_t && o < p.c_out;
-                const float* src = ok ? p.wt2 + static_cast<size_t>(o) * wpitch + c * 32 + q * 4 : p.wt2;
-                cp_async16(b_smem + row * 128 + ((q ^ (row & 7)) << 4), src, ok ? 16u : 0u);
-            }
-            cp_async_commit();
-            // signal the previous chunk once its copies have landed (one group stays in flight)
-            if (c > 0) {
-                cp_async_wait<1>();
-                fence_proxy_async();
-                mbar_arrive(smem_u32(&s_full[(c - 1) % NS]));
-            }
+            cp_async_wait<0>();
+            fence_proxy_async();
+            if (!aborted(abort_flag)) mbar_arrive(smem_u32(&s_full[(n_chunks - 1) % NS]));
         }
-        cp_async_wait<0>();
-        fence_proxy_async();
-        if (!aborted(abort_flag)) mbar_arrive(smem_u32(&s_full[(n_chunks - 1) % NS]));
     } else if (warp < 4) {
         // =========================== compactors, then epilogue ===========================
         const int row = tid;  // TMEM lane = pixel row
         const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+        const uint32_t rx4 = static_cast<uint32_t>(row & 7) << 4;
         const size_t rpitch = static_cast<size_t>(n_chunks) * 32;
         int use = 0;  // running count of operand-buffer uses
         for (int c = 0; c < n_chunks && !aborted(abort_flag); ++c) {
             const int s = c % NS;
-            const uint32_t slab_row = ring + s * cfg.stage_bytes + cfg.b_bytes + static_cast<uint32_t>(row * cfg.slab_pitch) * 4u;
+            const uint32_t slab_row = ring + s * cfg.stage_bytes + cfg.b_bytes + row * 128;
             for (int t = 0; t < g_here; ++t, ++use) {
                 // kept-column offsets of this (tile, chunk): warp-uniform, fetched before the waits
                 uint32_t relw[KC / 4];
                 const uint32_t* rp = reinterpret_cast<const uint32_t*>(p.rel2 + static_cast<size_t>(tile0 + t) * rpitch + c * 32);
 #pragma unroll
                 for (int q = 0; q < KC / 4; ++q) relw[q] = __ldg(rp + q);
-                // (the vote keeps the warp together for the .sync.aligned TMEM stores that follow)
+                // (the votes keep the warp together for the .sync.aligned TMEM stores that follow)
                 bool ok = t != 0 || mbar_wait(smem_u32(&s_full[s]), (c / NS) & 1);
                 if (!__all_sync(0xFFFFFFFFu, ok)) { *abort_flag = 3; break; }
                 const int buf = use % NA;
@@ -182,8 +234,10 @@ __global__ void __launch_bounds__(288, 2) k_conv_slab(const ConvParams p, const 
 #pragma unroll
                 for (int j = 0; j < KC; ++j) {
                     const uint32_t rel = (relw[j >> 2] >> ((j & 3) * 8)) & 0xFFu;
+                    // sub-tile (rel / 32), 16-byte piece ((rel / 4) % 8) ^ (row % 8), word rel % 4
+                    const uint32_t u = ((rel & 31u) << 2) + ((rel >> 5) * SUB_BYTES);
                     float f;
-                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(f) : "r"(slab_row + rel * 4u));
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(f) : "r"(slab_row + (u ^ rx4)));
                     v[j] = __float_as_uint(to_tf32(f));
                 }
                 const uint32_t a_addr = tmem + lane_addr + MAX_BN_COLS + buf * 32;
@@ -253,7 +307,7 @@ __global__ void __launch_bounds__(288, 2) k_conv_slab(const ConvParams p, const 
                 const int buf = use % NA;
                 if (!mbar_wait(smem_u32(&s_aready[buf]), (use / NA) & 1)) { *abort_flag = 7; break; }
                 tc_fence_after();
-                const uint64_t bdesc = umma_desc_k_sw128(b_smem + t * cfg.umma_n * 128, 1024);
+                const uint64_t bdesc = umma_desc_k_sw128(b_smem + t * cfg.b_tile_rows * 128, 1024);
                 const uint32_t a_addr = tmem + MAX_BN_COLS + buf * 32;
 #pragma unroll
                 for (int kq = 0; kq < KC / 8; ++kq)
@@ -277,6 +331,76 @@ __global__ void __launch_bounds__(288, 2) k_conv_slab(const ConvParams p, const 
     if (warp == 8) tmem_dealloc(tmem, TMEM_COLS);
 }
 
+// ---- tensor maps -----------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+std::once_flag g_encode_once;
+
+bool load_encoders()
+{
+    std::call_once(g_encode_once, [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            g_encode_tiled = reinterpret_cast<EncodeTiledFn>(f);
+        f = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(f);
+        (void)cudaGetLastError();
+    });
+    return g_encode_tiled && g_encode_im2col;
+}
+
+// Activations as an im2col tensor map: NHWC seen as (C, W, H, N); the box is 32 channels x 128
+// output pixels; the base-pixel window runs from -pad to pad - (K - 1) * dil in each direction
+// and is walked with the convolution stride.
+bool encode_x_map(const ConvParams& p, CUtensorMap* tm)
+{
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.c_in), static_cast<cuuint64_t>(p.w),
+                                static_cast<cuuint64_t>(p.h), static_cast<cuuint64_t>(p.batch)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(p.c_in) * 4, static_cast<cuuint64_t>(p.w) * p.c_in * 4,
+                                   static_cast<cuuint64_t>(p.h) * p.w * p.c_in * 4};
+    const int lower[2] = {-p.pad_w, -p.pad_h};
+    const int upper[2] = {p.pad_w - (p.kw - 1) * p.dil_w, p.pad_h - (p.kh - 1) * p.dil_h};
+    const cuuint32_t trav[4] = {1, static_cast<cuuint32_t>(p.stride_w), static_cast<cuuint32_t>(p.stride_h), 1};
+    return g_encode_im2col(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(p.x), dims, strides, lower, upper,
+                           32, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Chunk-major weights [c_out][chunks * 32] as a tiled map with a 32 x rows box.
+bool encode_w_map(const ConvParams& p, int rows, CUtensorMap* tm)
+{
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.v2_chunks) * 32, static_cast<cuuint64_t>(p.c_out)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(p.v2_chunks) * 32 * 4};
+    const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(rows)};
+    const cuuint32_t es[2] = {1, 1};
+    return g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(p.wt2), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tma_admissible(const ConvParams& p)
+{
+    if (p.c_in % 32 != 0 || p.tile_t % 8 != 0) return false;
+    // im2col maps of very small tensors are not used: the cp.async path takes them
+    if (static_cast<long long>(p.batch) * p.h * p.w * p.c_in * 4 < 131072) return false;
+    if (p.pad_w > 127 || p.pad_h > 127) return false;
+    if ((p.kw - 1) * p.dil_w - p.pad_w > 128 || (p.kh - 1) * p.dil_h - p.pad_h > 128) return false;
+    if ((p.kw - 1) * p.dil_w > 65535 || (p.kh - 1) * p.dil_h > 65535) return false;
+    if (p.stride_w > 8 || p.stride_h > 8) return false;
+    return load_encoders();
+}
+
 bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SlabCfg* cfg)
 {
     if (!p.wt2 || !p.rel2) return false;
@@ -291,13 +415,16 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SlabCfg* cfg)
         if (g < 1 || g * umma_n > MAX_BN_COLS) return false;
     }
     g = g < p.n_tiles ? g : p.n_tiles;
+    cfg->use_tma = tma_admissible(p) && !(plan && plan->split == 1) ? 1 : 0;  // split = 1 forces the cp.async producer
     cfg->g_tiles = g;
     cfg->umma_n = umma_n;
     cfg->n_slices = (p.n_tiles + g - 1) / g;
-    cfg->slab_pitch = p.v2_s + 1 + (p.v2_s % 2);  // odd number of words
-    cfg->slab_bytes = ((BM * cfg->slab_pitch * 4 + 1023) / 1024) * 1024;
-    cfg->b_bytes = g * umma_n * 128;                // multiple of 2048
-    cfg->stage_bytes = cfg->slab_bytes + cfg->b_bytes;
+    cfg->segs = (p.v2_s + 31) / 32;
+    cfg->b_tile_rows = cfg->use_tma ? p.tile_t : umma_n;
+    cfg->b_rows = g * cfg->b_tile_rows;
+    // room for the MMA of the last tile to read umma_n rows; whole 1024-byte swizzle atoms
+    cfg->b_bytes = ((((g - 1) * cfg->b_tile_rows + umma_n) * 128 + 1023) / 1024) * 1024;
+    cfg->stage_bytes = cfg->segs * SUB_BYTES + cfg->b_bytes;
     const int budget = 110 * 1024;                  // two CTAs per SM
     int stages = plan && plan->stages > 0 ? plan->stages : 3;
     if (stages > NSTAGE_MAX) return false;
@@ -307,21 +434,33 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SlabCfg* cfg)
     return true;
 }
 
-template <int KC>
+template <int KC, bool TMA>
 nm_status_t launch(const ConvParams& p, const SlabCfg& cfg, cudaStream_t st)
 {
+    alignas(64) CUtensorMap tm_x, tm_w;
+    memset(&tm_x, 0, sizeof(tm_x));
+    memset(&tm_w, 0, sizeof(tm_w));
+    if (TMA && (!encode_x_map(p, &tm_x) || !encode_w_map(p, cfg.b_rows, &tm_w)))
+        return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed");
     size_t smem = static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 1024;
     if (smem < 78 * 1024) smem = 78 * 1024;  // never more than two CTAs (2 x 256 TMEM columns) per SM
-    cudaError_t e = cudaFuncSetAttribute(k_conv_slab<KC>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    cudaError_t e = cudaFuncSetAttribute(k_conv_slab<KC, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 2): %s", cudaGetErrorString(e));
     const long long tiles_m = (p.pixels + BM - 1) / BM;
     const long long blocks = tiles_m * cfg.n_slices;
     if (blocks > 0x7FFFFFFFll) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: too many output tiles");
-    k_conv_slab<KC><<<static_cast<unsigned>(blocks), 288, smem, st>>>(p, cfg);
+    k_conv_slab<KC, TMA><<<static_cast<unsigned>(blocks), 288, smem, st>>>(p, cfg, tm_x, tm_w);
     nmhost::count_launch(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_conv2d launch (variant 2): %s", cudaGetErrorString(e));
     return NM_OK;
+}
+
+template <int KC>
+nm_status_t launch_kc(const ConvParams& p, const SlabCfg& cfg, cudaStream_t st)
+{
+    return cfg.use_tma ? launch<KC, true>(p, cfg, st) : launch<KC, false>(p, cfg, st);
 }
 
 }  // namespace
@@ -339,10 +478,10 @@ nm_status_t launch_conv_slab(const ConvParams& p, const nm_plan_t* plan, cudaStr
     SlabCfg cfg;
     if (!make_cfg(p, plan, &cfg)) return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the slab kernel does not take this layer / plan");
     switch (p.v2_kc) {
-        case 8: return launch<8>(p, cfg, st);
-        case 16: return launch<16>(p, cfg, st);
-        case 24: return launch<24>(p, cfg, st);
-        case 32: return launch<32>(p, cfg, st);
+        case 8: return launch_kc<8>(p, cfg, st);
+        case 16: return launch_kc<16>(p, cfg, st);
+        case 24: return launch_kc<24>(p, cfg, st);
+        case 32: return launch_kc<32>(p, cfg, st);
     }
     return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unsupported kept-columns-per-chunk %d", p.v2_kc);
 }

@@ -19,9 +19,9 @@ def nm():
 def _plans(nm, s):
     """Every kernel variant that admits the shape, plus the library default."""
     out = [None]
-    for variant in (1, 2):
+    for variant, split in ((1, 0), (2, 0), (2, 1)):   # split = 1: slab kernel with its cp.async producer
         p = nm.nm_plan_t()
-        p.variant = variant
+        p.variant, p.split = variant, split
         out.append(p)
     return out
 
@@ -78,6 +78,51 @@ SMALL = [
 @pytest.mark.parametrize("s", SMALL, ids=lambda s: s.name)
 def test_small_shapes(nm, s):
     _run(nm, s)
+
+
+# inputs of at least 128 KiB with c_in % 32 == 0: these take the TMA (im2col) producer
+MEDIUM = [
+    ConvShape("tma_3x3", 2, 16, 16, 64, 64, 3, 3, 1, 1, 1, 2, 4, 32),
+    ConvShape("tma_ragged_tail", 3, 13, 13, 64, 64, 3, 3, 1, 1, 1, 2, 4, 64),      # 507 pixels
+    ConvShape("tma_stride2", 2, 15, 15, 128, 64, 3, 3, 2, 1, 1, 2, 4, 32),
+    ConvShape("tma_dilation2", 1, 20, 20, 96, 32, 3, 3, 1, 2, 2, 2, 4, 32),
+    ConvShape("tma_1x1", 2, 14, 14, 256, 96, 1, 1, 1, 0, 1, 2, 4, 32),
+    ConvShape("tma_1x1_stride2", 2, 14, 14, 256, 64, 1, 1, 2, 0, 1, 1, 4, 64),
+    ConvShape("tma_5x5", 1, 24, 24, 64, 32, 5, 5, 1, 2, 1, 2, 8, 16),
+    ConvShape("tma_tile8", 2, 16, 16, 64, 24, 3, 3, 1, 1, 1, 2, 4, 8),
+    ConvShape("tma_1of8", 1, 16, 16, 128, 64, 3, 3, 1, 1, 1, 1, 8, 64),
+    ConvShape("tma_3of4", 1, 16, 16, 128, 64, 1, 1, 1, 0, 1, 3, 4, 64),
+    ConvShape("tma_dense", 1, 16, 16, 128, 48, 3, 3, 1, 1, 1, 4, 4, 16),
+    ConvShape("tma_tile128", 1, 16, 16, 128, 256, 3, 3, 1, 1, 1, 2, 4, 128),
+]
+
+
+@pytest.mark.parametrize("s", MEDIUM, ids=lambda s: s.name)
+def test_medium_shapes(nm, s):
+    _run(nm, s)
+
+
+@pytest.mark.parametrize("s", MEDIUM[:6], ids=lambda s: s.name)
+def test_medium_shapes_integer_exact(nm, s):
+    _run(nm, s, integer=True)
+
+
+def test_asymmetric_geometry(nm):
+    """3x5 kernel, stride (1, 2), padding (1, 2), dilation (2, 1): catches any h / w mix-up."""
+    import oracle
+    g = torch.Generator().manual_seed(77)
+    w = torch.randint(-3, 4, (32, 3, 5, 64), generator=g).float()
+    x = torch.randint(-3, 4, (2, 18, 22, 64), generator=g).float()
+    b = torch.randint(-3, 4, (32,), generator=g).float()
+    stride, pad, dil = (1, 2), (1, 2), (2, 1)
+    vr, ir = oracle.prune(w.numpy(), 2, 4, 16)
+    yr = oracle.conv2d(vr, ir, 3, 5, 64, 16, x.numpy(), stride, pad, dil, b.numpy(), True)
+    hnd = nm.nm_prune(w.cuda(), 2, 4, 16)
+    for plan in _plans(nm, None):
+        y = nm.nm_conv2d(hnd, x.cuda(), 3, 5, stride, pad, dil, b.cuda(), True, plan=plan)
+        nm.nm_weights_check(hnd)
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy(), yr), f"plan {plan.as_dict() if plan else None}"
 
 
 @pytest.mark.parametrize("s", SMALL[:8], ids=lambda s: s.name)
