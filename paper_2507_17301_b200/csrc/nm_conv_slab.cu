@@ -49,6 +49,7 @@ struct SlabCfg {
     int b_tile_rows;  // row distance between two tiles' weights in shared memory
     int b_bytes, stage_bytes;
     int use_tma;
+    int tma_store;    // epilogue through shared memory + TMA store
 };
 
 __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
@@ -65,7 +66,7 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const void* tma
 template <int KC, bool TMA>
 __global__ void __launch_bounds__(288, 2)
 k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUtensorMap tm_x,
-            const __grid_constant__ CUtensorMap tm_w)
+            const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[NSTAGE_MAX], s_free[NSTAGE_MAX], s_aready[NA], s_afree[NA], s_dready;
@@ -255,7 +256,47 @@ k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUten
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_dready), 0);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 5;
         }
-        if (!__any_sync(0xFFFFFFFFu, aborted(abort_flag))) {
+        if (cfg.tma_store) {
+            // coalesced path: 32-column blocks staged in the (now idle) ring in the swizzled layout
+            // a tiled TMA store expects, one 32 x 32 box per warp and block
+            if (!__any_sync(0xFFFFFFFFu, aborted(abort_flag))) {
+                tc_fence_after();
+                const int bn_cols = g_here * p.tile_t;          // contiguous: tile_t is a multiple of 16 here
+                const int o0 = tile0 * p.tile_t;
+                for (int blk = 0; blk * 32 < bn_cols; ++blk) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + blk * 32, v);
+                    tmem_ld_wait();
+                    const uint32_t stage_row = ring + blk * SUB_BYTES + row * 128;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float o[4];
+                        float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + q);
+                        o[0] = __uint_as_float(v[q * 4 + 0]) + bv.x;
+                        o[1] = __uint_as_float(v[q * 4 + 1]) + bv.y;
+                        o[2] = __uint_as_float(v[q * 4 + 2]) + bv.z;
+                        o[3] = __uint_as_float(v[q * 4 + 3]) + bv.w;
+                        if (p.relu) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
+                        }
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage_row + ((q ^ (row & 7)) << 4)),
+                                     "f"(o[0]), "f"(o[1]), "f"(o[2]), "f"(o[3])
+                                     : "memory");
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0 && pix0 + warp * 32 < p.pixels)
+                        tma_store_2d(&tm_y, ring + blk * SUB_BYTES + warp * 32 * 128, o0 + blk * 32,
+                                     static_cast<int>(pix0) + warp * 32);
+                }
+                if (lane == 0) {
+                    tma_store_commit();
+                    tma_store_wait_read();  // shared memory must outlive the stores' reads
+                }
+            }
+        } else if (!__any_sync(0xFFFFFFFFu, aborted(abort_flag))) {
             tc_fence_after();
             const long long pix = pix0 + row;
             float* yrow = p.y + static_cast<size_t>(pix < p.pixels ? pix : 0) * p.c_out;
@@ -389,6 +430,18 @@ bool encode_w_map(const ConvParams& p, int rows, CUtensorMap* tm)
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output [pixels][c_out] as a tiled map with a 32-channel x 32-pixel box (one warp's share).
+bool encode_y_map(const ConvParams& p, CUtensorMap* tm)
+{
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.c_out), static_cast<cuuint64_t>(p.pixels)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(p.c_out) * 4};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t es[2] = {1, 1};
+    return g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, p.y, dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool tma_admissible(const ConvParams& p)
 {
     if (p.c_in % 32 != 0 || p.tile_t % 8 != 0) return false;
@@ -431,17 +484,26 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SlabCfg* cfg)
     while (stages > 1 && stages * cfg->stage_bytes + 1024 > budget && !(plan && plan->stages > 0)) --stages;
     if (stages * cfg->stage_bytes + 1024 > 225 * 1024) return false;
     cfg->stages = stages;
+    // TMA-store epilogue: channel blocks of 32 must tile the CTA's channel range exactly, the
+    // staging blocks must fit the ring, and the pixel count must fit the map's 32-bit coordinate
+    const int bn_cols = g * p.tile_t;
+    cfg->tma_store = load_encoders() && p.tile_t % 16 == 0 && bn_cols % 32 == 0 && p.c_out % 4 == 0 &&
+                     (bn_cols / 32) * SUB_BYTES <= stages * cfg->stage_bytes && p.pixels < (1ll << 31) &&
+                     p.n_tiles % g == 0 && p.c_out % p.tile_t == 0 && !(plan && plan->split == 2);
     return true;
 }
 
 template <int KC, bool TMA>
 nm_status_t launch(const ConvParams& p, const SlabCfg& cfg, cudaStream_t st)
 {
-    alignas(64) CUtensorMap tm_x, tm_w;
+    alignas(64) CUtensorMap tm_x, tm_w, tm_y;
     memset(&tm_x, 0, sizeof(tm_x));
     memset(&tm_w, 0, sizeof(tm_w));
+    memset(&tm_y, 0, sizeof(tm_y));
     if (TMA && (!encode_x_map(p, &tm_x) || !encode_w_map(p, cfg.b_rows, &tm_w)))
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed");
+    if (cfg.tma_store && !encode_y_map(p, &tm_y))
+        return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: output tensor-map encoding failed");
     size_t smem = static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 1024;
     if (smem < 78 * 1024) smem = 78 * 1024;  // never more than two CTAs (2 x 256 TMEM columns) per SM
     cudaError_t e = cudaFuncSetAttribute(k_conv_slab<KC, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -450,7 +512,7 @@ nm_status_t launch(const ConvParams& p, const SlabCfg& cfg, cudaStream_t st)
     const long long tiles_m = (p.pixels + BM - 1) / BM;
     const long long blocks = tiles_m * cfg.n_slices;
     if (blocks > 0x7FFFFFFFll) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: too many output tiles");
-    k_conv_slab<KC, TMA><<<static_cast<unsigned>(blocks), 288, smem, st>>>(p, cfg, tm_x, tm_w);
+    k_conv_slab<KC, TMA><<<static_cast<unsigned>(blocks), 288, smem, st>>>(p, cfg, tm_x, tm_w, tm_y);
     nmhost::count_launch(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_conv2d launch (variant 2): %s", cudaGetErrorString(e));
