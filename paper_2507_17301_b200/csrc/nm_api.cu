@@ -33,6 +33,7 @@ void free_handle_memory(nm_weights* h)
     cudaFree(h->status);
     cudaFree(h->wt2);
     cudaFree(h->rel2);
+    cudaFree(h->wx);
     h->magic = 0;
     delete h;
 }
@@ -118,6 +119,7 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     p->wt2 = w->v2_ok ? w->wt2 : nullptr;
     p->rel2 = w->v2_ok ? w->rel2 : nullptr;
     p->v2_kc = w->v2_kc; p->v2_s = w->v2_s; p->v2_chunks = w->v2_chunks;
+    p->wx = w->wx;
     return NM_OK;
 }
 
@@ -126,12 +128,17 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
     const int variant = plan ? plan->variant : 0;
     switch (variant) {
         case 0:
+            if (nmhost::stream_plan_ok(p, nullptr)) return nmhost::launch_conv_stream(p, nullptr, st);
             if (nmhost::slab_plan_ok(p, nullptr)) return nmhost::launch_conv_slab(p, nullptr, st);
             return nmhost::launch_conv_gather(p, st);
         case 1:
             return nmhost::launch_conv_gather(p, st);
         case 2:
             return nmhost::launch_conv_slab(p, plan, st);
+        case 3:
+            return nmhost::launch_conv_stream(p, plan, st);
+        case 4:
+            return nmhost::launch_conv_expand(p, plan, st);
         default:
             return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
     }
@@ -142,6 +149,16 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
 {
     std::vector<nm_plan_t> out;
     nm_plan_t a;
+    std::memset(&a, 0, sizeof(a));
+    for (int bn : {64, 128, 256}) {         // expanded-operand kernel
+        a.variant = 4; a.bn = bn; a.stages = 0;
+        if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);
+    }
+    std::memset(&a, 0, sizeof(a));
+    for (int bn : {0, 256, p.tile_t}) {     // stream kernel: default width, widest, one tile per CTA
+        a.variant = 3; a.bn = bn; a.stages = 0;
+        if ((bn == 0 || bn != p.tile_t || bn < 128) && nmhost::stream_plan_ok(p, &a)) out.push_back(a);
+    }
     std::memset(&a, 0, sizeof(a));
     for (int bn : {0, p.tile_t}) {          // default (as many tiles as fit) and one tile per CTA
         for (int stages : {2, 3}) {
@@ -180,6 +197,7 @@ nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, 
     if (s != NM_OK) return s;
     s = nmhost::prune_on_device(w_dense, h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_expanded_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         return s;
@@ -197,6 +215,7 @@ nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int 
     if (s != NM_OK) return s;
     s = nmhost::build_from_compressed(values, indices, h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_expanded_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         *out = nullptr;

@@ -1,0 +1,314 @@
+// Variant 4: expanded-operand kernel — persistent implicit GEMM that feeds the tensor core the
+// DENSE activation slab straight from shared memory and lets zero weights stand for the pruned
+// columns.
+//
+// Nothing is compacted: the slab [128 pixels x 32 source columns] that TMA's im2col mode lays
+// down in the 128-byte-swizzled K-major layout IS the A operand, and the B operand is the pruned
+// weight matrix re-expanded to its dense [channels x K] shape (TF32, zeros in the pruned
+// columns, built once per handle).  The tensor core therefore spends M/N times the kept FLOPs,
+// but no thread ever touches an activation.  It moves the same HBM bytes as the gathering
+// kernels (with N:M groups along the channel axis every 16-byte vector holds survivors, so a
+// gather cannot skip input bytes either), which makes it the right choice wherever the layer is
+// bound by HBM and the tensor pipe has slack; the auto-tuner decides per layer by measurement.
+// The pruning tile width plays no role here, so any tile_t is accepted.
+//
+//   producer (1 thread)   TMA im2col load of the slab + tiled load of the weight block per stage
+//   MMA issuer (1 thread) four 128 x BN x 8 TF32 tcgen05.mma (SS) per stage into one of two
+//                         accumulator buffers in tensor memory
+//   epilogue (8 warps)    TMEM -> registers, + bias, ReLU, swizzled staging, TMA store to NHWC;
+//                         overlaps the next work item's main loop
+// Work items (128 pixels x BN channels) are walked in a static persistent schedule; every wait is
+// bounded and reports through the handle's status word.
+#include "nm_internal.h"
+#include "nm_ptx.cuh"
+#include "nm_tmap.cuh"
+
+namespace {
+
+using namespace nmk;
+
+constexpr int BM = 128;
+constexpr int SUB_BYTES = BM * 128;
+constexpr int NSTAGE_MAX = 8;
+constexpr int THREADS = 384;                   // 4 service warps + 8 epilogue warps
+constexpr int STAGING_BYTES = 8 * 2 * 4096;    // per epilogue warp two 32 x 32 output boxes
+
+struct ExpandCfg {
+    int bn;           // output channels per work item
+    int n_slices;
+    int stages;
+    int b_bytes;      // weight bytes per stage (bn rows of 128 bytes)
+    int stage_bytes;
+    int n_sub;        // K / 32
+    long long n_work;
+};
+
+__device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
+
+__global__ void __launch_bounds__(THREADS, 1)
+k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ CUtensorMap tm_x,
+              const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t s_full[NSTAGE_MAX], s_free[NSTAGE_MAX], s_accfull[2], s_accfree[2];
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NS = cfg.stages, n_sub = cfg.n_sub;
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t staging = ring + NS * cfg.stage_bytes;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == 2) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (tid == 0) {
+        for (int i = 0; i < NSTAGE_MAX; ++i) {
+            mbar_init(smem_u32(&s_full[i]), 1);   // producer's expect-tx arrival
+            mbar_init(smem_u32(&s_free[i]), 1);   // MMA commit
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&s_accfull[i]), 1);   // MMA commit
+            mbar_init(smem_u32(&s_accfree[i]), 8);   // epilogue warps
+        }
+        mbar_fence_init();
+        s_abort = 0;
+        tma_prefetch_desc(&tm_x);
+        tma_prefetch_desc(&tm_w);
+        tma_prefetch_desc(&tm_y);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+
+    if (warp == 0) {
+        // =========================== producer ===========================
+        if (lane == 0) {
+            const int hw = p.ho * p.wo;
+            const uint32_t tx = SUB_BYTES + static_cast<uint32_t>(cfg.bn) * 128u;
+            long long cc = 0;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+                const int slice = static_cast<int>(work % cfg.n_slices);
+                const long long pix0 = (work / cfg.n_slices) * BM;
+                const int n0 = static_cast<int>(pix0 / hw);
+                const int rem = static_cast<int>(pix0 - static_cast<long long>(n0) * hw);
+                const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
+                const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
+                int tap = 0, ch = 0;
+                for (int c = 0; c < n_sub; ++c, ++cc) {
+                    const int s = static_cast<int>(cc % NS);
+                    if (cc >= NS && !mbar_wait(smem_u32(&s_free[s]), static_cast<uint32_t>((cc / NS) - 1) & 1u))
+                        *abort_flag = 2;
+                    if (aborted(abort_flag)) break;
+                    const uint32_t a_smem = ring + s * cfg.stage_bytes;
+                    const uint32_t bar = smem_u32(&s_full[s]);
+                    mbar_arrive_expect_tx(bar, tx);
+                    tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>((tap % p.kw) * p.dil_w),
+                                       static_cast<uint16_t>((tap / p.kw) * p.dil_h));
+                    tma_load_2d(a_smem + SUB_BYTES, &tm_w, bar, c * 32, slice * cfg.bn);
+                    ch += 32;
+                    if (ch >= p.c_in) { ch = 0; ++tap; }
+                }
+            }
+            if (aborted(abort_flag)) {
+                for (long long back = 1; back <= NS && back <= cc; ++back) {
+                    const long long cl = cc - back;
+                    (void)mbar_wait(smem_u32(&s_full[cl % NS]), static_cast<uint32_t>(cl / NS) & 1u);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
+            long long cc = 0, ti = 0;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x, ++ti) {
+                const int ab = static_cast<int>(ti & 1);
+                if (ti >= 2 && !mbar_wait(smem_u32(&s_accfree[ab]), static_cast<uint32_t>((ti >> 1) - 1) & 1u)) {
+                    *abort_flag = 5;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t acc = tmem + ab * cfg.bn;
+                for (int c = 0; c < n_sub; ++c, ++cc) {
+                    const int s = static_cast<int>(cc % NS);
+                    if (!mbar_wait(smem_u32(&s_full[s]), static_cast<uint32_t>(cc / NS) & 1u)) { *abort_flag = 6; break; }
+                    tc_fence_after();
+                    const uint32_t a_smem = ring + s * cfg.stage_bytes;
+                    const uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
+                    const uint64_t bdesc = umma_desc_k_sw128(a_smem + SUB_BYTES, 1024);
+#pragma unroll
+                    for (int kq = 0; kq < 4; ++kq)
+                        umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > 0 || kq > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(&s_free[s]));
+                }
+                if (aborted(abort_flag)) break;
+                umma_commit(smem_u32(&s_accfull[ab]));
+            }
+        }
+    } else if (warp >= 4) {
+        // =========================== epilogue ===========================
+        const int q = warp & 3;            // TMEM lane quadrant
+        const int half = (warp - 4) >> 2;  // which channel blocks of 32: blk = 2 * i + half
+        const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+        const uint32_t my_staging = staging + (warp - 4) * 2 * 4096;
+        const uint32_t rx = static_cast<uint32_t>(lane & 7);
+        const int n_blk = cfg.bn / 32;
+        long long ti = 0;
+        uint32_t nb = 0;
+        for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
+            const int slice = static_cast<int>(work % cfg.n_slices);
+            const long long pix0 = (work / cfg.n_slices) * BM;
+            const int ab = static_cast<int>(ti & 1);
+            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), static_cast<uint32_t>(ti >> 1) & 1u);
+            if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
+            if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
+            tc_fence_after();
+            const int o0 = slice * cfg.bn;
+            for (int blk = half; blk < n_blk; blk += 2, ++nb) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_addr + ab * cfg.bn + blk * 32, v);
+                tmem_ld_wait();
+                if (blk + 2 >= n_blk) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+                }
+                const uint32_t box = my_staging + (nb & 1u) * 4096;
+                if (lane == 0 && nb >= 2) tma_store_wait_read_n<1>();
+                __syncwarp();
+                const uint32_t stage_row = box + lane * 128;
+#pragma unroll
+                for (int qq = 0; qq < 8; ++qq) {
+                    float o[4];
+                    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
+                    o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
+                    o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
+                    o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
+                    o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
+                    if (p.relu) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
+                    }
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage_row + ((qq ^ rx) << 4)), "f"(o[0]),
+                                 "f"(o[1]), "f"(o[2]), "f"(o[3])
+                                 : "memory");
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    if (pix0 + q * 32 < p.pixels)
+                        tma_store_2d(&tm_y, box, o0 + blk * 32, static_cast<int>(pix0) + q * 32);
+                    tma_store_commit();
+                }
+            }
+            if (n_blk == 1 && half == 1) {
+                // a single channel block: the second warp of the quadrant only releases the buffer
+                if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && s_abort != 0) {
+        atomicExch(p.status + 0, static_cast<int>(NM_ERR_TIMEOUT));
+        atomicExch(p.status + 1, 40 + s_abort);
+        atomicExch(p.status + 2, static_cast<int>(blockIdx.x));
+    }
+    if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            n = 148;
+    }
+    return n;
+}
+
+bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
+{
+    if (!p.wx || !nmtm::available()) return false;
+    if (p.c_in % 32 != 0 || p.c_out % 32 != 0) return false;
+    if (!nmtm::im2col_geometry_ok(p)) return false;
+    if (static_cast<long long>(p.batch) * p.h * p.w * p.c_in * 4 < 131072) return false;
+    if (p.pixels >= (1ll << 31) - BM) return false;
+    int bn = 0;
+    if (plan && plan->bn > 0) {
+        bn = plan->bn;
+    } else {
+        for (int cand : {128, 256, 64, 96, 32, 160, 192, 224})
+            if (cand <= p.c_out && p.c_out % cand == 0) { bn = cand; break; }
+    }
+    if (bn < 32 || bn > 256 || bn % 32 != 0 || p.c_out % bn != 0) return false;
+    cfg->bn = bn;
+    cfg->n_slices = p.c_out / bn;
+    cfg->b_bytes = ((bn * 128 + 1023) / 1024) * 1024;
+    cfg->stage_bytes = SUB_BYTES + cfg->b_bytes;
+    cfg->n_sub = p.k / 32;
+    const int budget = 227 * 1024 - 1024 - STAGING_BYTES - 1024;
+    int stages = plan && plan->stages > 0 ? plan->stages : NSTAGE_MAX;
+    if (stages > NSTAGE_MAX) return false;
+    if (plan && plan->stages > 0) {
+        if (stages * cfg->stage_bytes > budget) return false;
+    } else {
+        while (stages > 2 && stages * cfg->stage_bytes > budget) --stages;
+        if (stages * cfg->stage_bytes > budget) return false;
+    }
+    cfg->stages = stages;
+    cfg->n_work = ((p.pixels + BM - 1) / BM) * cfg->n_slices;
+    return true;
+}
+
+// Dense [c_out][K] weights as a tiled map with a 32-column x `rows` box.
+bool encode_wx(const ConvParams& p, int rows, CUtensorMap* tm)
+{
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.k), static_cast<cuuint64_t>(p.c_out)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(p.k) * 4};
+    const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(rows)};
+    const cuuint32_t es[2] = {1, 1};
+    return nmtm::encoders().tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(p.wx), dims, strides, box,
+                                  es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+namespace nmhost {
+
+bool expand_plan_ok(const ConvParams& p, const nm_plan_t* plan)
+{
+    ExpandCfg cfg;
+    return make_cfg(p, plan, &cfg);
+}
+
+nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st)
+{
+    ExpandCfg cfg;
+    if (!make_cfg(p, plan, &cfg))
+        return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the expanded-operand kernel does not take this layer / plan");
+    alignas(64) CUtensorMap tm_x, tm_w, tm_y;
+    if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !encode_wx(p, cfg.bn, &tm_w) || !nmtm::encode_y_tiled(p, &tm_y))
+        return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 4)");
+    size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + STAGING_BYTES;
+    if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
+    cudaError_t e = cudaFuncSetAttribute(k_conv_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
+    const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
+    k_conv_expand<<<static_cast<unsigned>(grid), THREADS, smem, st>>>(p, cfg, tm_x, tm_w, tm_y);
+    count_launch(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 4): %s", cudaGetErrorString(e));
+    return NM_OK;
+}
+
+}  // namespace nmhost

@@ -21,12 +21,9 @@
 // Epilogue (the compactor warps): TMEM -> registers, + bias, ReLU, NHWC store.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, reports through the
 // status word and drains to the common exit where TMEM is released.
-#include <cuda.h>
-
-#include <mutex>
-
 #include "nm_internal.h"
 #include "nm_ptx.cuh"
+#include "nm_tmap.cuh"
 
 namespace {
 
@@ -53,15 +50,6 @@ struct SlabCfg {
 };
 
 __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
-
-__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const void* tmap, uint32_t bar, int c, int w, int h,
-                                                   int n, uint16_t off_w, uint16_t off_h)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cta.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
-        : "memory");
-}
 
 template <int KC, bool TMA>
 __global__ void __launch_bounds__(288, 2)
@@ -372,86 +360,13 @@ k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUten
     if (warp == 8) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-// ---- tensor maps -----------------------------------------------------------------------------------
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
-                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                    CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode_tiled = nullptr;
-EncodeIm2colFn g_encode_im2col = nullptr;
-std::once_flag g_encode_once;
-
-bool load_encoders()
-{
-    std::call_once(g_encode_once, [] {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            g_encode_tiled = reinterpret_cast<EncodeTiledFn>(f);
-        f = nullptr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(f);
-        (void)cudaGetLastError();
-    });
-    return g_encode_tiled && g_encode_im2col;
-}
-
-// Activations as an im2col tensor map: NHWC seen as (C, W, H, N); the box is 32 channels x 128
-// output pixels; the base-pixel window runs from -pad to pad - (K - 1) * dil in each direction
-// and is walked with the convolution stride.
-bool encode_x_map(const ConvParams& p, CUtensorMap* tm)
-{
-    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.c_in), static_cast<cuuint64_t>(p.w),
-                                static_cast<cuuint64_t>(p.h), static_cast<cuuint64_t>(p.batch)};
-    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(p.c_in) * 4, static_cast<cuuint64_t>(p.w) * p.c_in * 4,
-                                   static_cast<cuuint64_t>(p.h) * p.w * p.c_in * 4};
-    const int lower[2] = {-p.pad_w, -p.pad_h};
-    const int upper[2] = {p.pad_w - (p.kw - 1) * p.dil_w, p.pad_h - (p.kh - 1) * p.dil_h};
-    const cuuint32_t trav[4] = {1, static_cast<cuuint32_t>(p.stride_w), static_cast<cuuint32_t>(p.stride_h), 1};
-    return g_encode_im2col(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(p.x), dims, strides, lower, upper,
-                           32, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// Chunk-major weights [c_out][chunks * 32] as a tiled map with a 32 x rows box.
-bool encode_w_map(const ConvParams& p, int rows, CUtensorMap* tm)
-{
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.v2_chunks) * 32, static_cast<cuuint64_t>(p.c_out)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(p.v2_chunks) * 32 * 4};
-    const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(rows)};
-    const cuuint32_t es[2] = {1, 1};
-    return g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(p.wt2), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// Output [pixels][c_out] as a tiled map with a 32-channel x 32-pixel box (one warp's share).
-bool encode_y_map(const ConvParams& p, CUtensorMap* tm)
-{
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.c_out), static_cast<cuuint64_t>(p.pixels)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(p.c_out) * 4};
-    const cuuint32_t box[2] = {32, 32};
-    const cuuint32_t es[2] = {1, 1};
-    return g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, p.y, dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
+// ---- launch configuration --------------------------------------------------------------------------
 bool tma_admissible(const ConvParams& p)
 {
     if (p.c_in % 32 != 0 || p.tile_t % 8 != 0) return false;
     // im2col maps of very small tensors are not used: the cp.async path takes them
     if (static_cast<long long>(p.batch) * p.h * p.w * p.c_in * 4 < 131072) return false;
-    if (p.pad_w > 127 || p.pad_h > 127) return false;
-    if ((p.kw - 1) * p.dil_w - p.pad_w > 128 || (p.kh - 1) * p.dil_h - p.pad_h > 128) return false;
-    if ((p.kw - 1) * p.dil_w > 65535 || (p.kh - 1) * p.dil_h > 65535) return false;
-    if (p.stride_w > 8 || p.stride_h > 8) return false;
-    return load_encoders();
+    return nmtm::im2col_geometry_ok(p) && nmtm::available();
 }
 
 bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SlabCfg* cfg)
@@ -487,7 +402,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SlabCfg* cfg)
     // TMA-store epilogue: channel blocks of 32 must tile the CTA's channel range exactly, the
     // staging blocks must fit the ring, and the pixel count must fit the map's 32-bit coordinate
     const int bn_cols = g * p.tile_t;
-    cfg->tma_store = load_encoders() && p.tile_t % 16 == 0 && bn_cols % 32 == 0 && p.c_out % 4 == 0 &&
+    cfg->tma_store = nmtm::available() && p.tile_t % 16 == 0 && bn_cols % 32 == 0 && p.c_out % 4 == 0 &&
                      (bn_cols / 32) * SUB_BYTES <= stages * cfg->stage_bytes && p.pixels < (1ll << 31) &&
                      p.n_tiles % g == 0 && p.c_out % p.tile_t == 0 && !(plan && plan->split == 2);
     return true;
@@ -500,9 +415,9 @@ nm_status_t launch(const ConvParams& p, const SlabCfg& cfg, cudaStream_t st)
     memset(&tm_x, 0, sizeof(tm_x));
     memset(&tm_w, 0, sizeof(tm_w));
     memset(&tm_y, 0, sizeof(tm_y));
-    if (TMA && (!encode_x_map(p, &tm_x) || !encode_w_map(p, cfg.b_rows, &tm_w)))
+    if (TMA && (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_w_tiled(p, cfg.b_rows, &tm_w)))
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed");
-    if (cfg.tma_store && !encode_y_map(p, &tm_y))
+    if (cfg.tma_store && !nmtm::encode_y_tiled(p, &tm_y))
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: output tensor-map encoding failed");
     size_t smem = static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 1024;
     if (smem < 78 * 1024) smem = 78 * 1024;  // never more than two CTAs (2 x 256 TMEM columns) per SM

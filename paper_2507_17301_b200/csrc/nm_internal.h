@@ -27,6 +27,8 @@ struct nm_weights {
     int v2_ok, v2_g, v2_kc, v2_s, v2_chunks;
     float* wt2;          // [c_out][v2_chunks * 32] TF32 weights, chunk-major, first v2_kc of each 32 used
     uint8_t* rel2;       // [n_tiles][v2_chunks * 32] source column of each kept column, relative to its chunk
+    // Expanded layout (variant 4): the pruned matrix back in dense shape, zeros in the pruned columns.
+    float* wx;           // [c_out][k] TF32, or NULL when the layer shape rules the variant out
 };
 
 // Geometry handed to the convolution kernels.
@@ -48,6 +50,8 @@ struct ConvParams {
     const float* wt2;
     const uint8_t* rel2;
     int v2_kc, v2_s, v2_chunks;
+    // expanded layout (variant 4)
+    const float* wx;
 };
 
 namespace nmhost {
@@ -60,6 +64,7 @@ nm_status_t prune_on_device(const float* w_dense, nm_weights* h, cudaStream_t st
 nm_status_t build_from_compressed(const float* values, const uint16_t* indices, nm_weights* h, cudaStream_t st);
 
 nm_status_t build_slab_layout(nm_weights* h, cudaStream_t st);
+nm_status_t build_expanded_layout(nm_weights* h, cudaStream_t st);
 
 // nm_conv_gather.cu — variant 1
 nm_status_t launch_conv_gather(const ConvParams& p, cudaStream_t st);
@@ -67,4 +72,12 @@ nm_status_t launch_conv_gather(const ConvParams& p, cudaStream_t st);
 // nm_conv_slab.cu — variant 2
 bool slab_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_slab(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
+// nm_conv_expand.cu — variant 4
+bool expand_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
+// nm_conv_stream.cu — variant 3
+bool stream_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_stream(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 }  // namespace nmhost

@@ -120,6 +120,17 @@ __global__ void k_build_slab(const float* __restrict__ values, const uint16_t* _
     if (o == r * tile_t) rel2[static_cast<size_t>(r) * pitch + chunk * 32 + jj] = static_cast<uint8_t>(col - chunk * s_cols);
 }
 
+// Expanded layout: wx[o][indices[o / T][j]] = TF32(values[o][j]); the rest stays zero.
+__global__ void k_expand(const float* __restrict__ values, const uint16_t* __restrict__ indices, int k, int kk,
+                         int tile_t, float* __restrict__ wx)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int o = blockIdx.y;
+    if (j >= kk) return;
+    const int col = indices[static_cast<size_t>(o / tile_t) * kk + j];
+    wx[static_cast<size_t>(o) * k + col] = nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
+}
+
 // Import path: every index row must be strictly ascending and below k.
 __global__ void k_check_indices(const uint16_t* __restrict__ indices, int kk, int k, int* __restrict__ bad)
 {
@@ -203,6 +214,27 @@ nm_status_t build_slab_layout(nm_weights* h, cudaStream_t st)
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "slab layout kernel: %s", cudaGetErrorString(e));
     h->v2_ok = 1;
+    return NM_OK;
+}
+
+nm_status_t build_expanded_layout(nm_weights* h, cudaStream_t st)
+{
+    h->wx = nullptr;
+    // only shapes the expanded-operand kernel takes: whole 32-column slabs, 32-channel output blocks
+    if (h->c_in % 32 != 0 || h->c_out % 32 != 0 || h->kk == 0) return NM_OK;
+    const size_t bytes = static_cast<size_t>(h->c_out) * h->k * sizeof(float);
+    if (cudaMalloc(&h->wx, bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        h->wx = nullptr;
+        return fail(NM_ERR_ALLOC, "cannot allocate the expanded weights (%zu bytes)", bytes);
+    }
+    cudaError_t e = cudaMemsetAsync(h->wx, 0, bytes, st);
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "expanded layout memset: %s", cudaGetErrorString(e));
+    const dim3 grid((h->kk + 127) / 128, h->c_out);
+    k_expand<<<grid, 128, 0, st>>>(h->values, h->indices, h->k, h->kk, h->tile_t, h->wx);
+    count_launch(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "expanded layout kernel: %s", cudaGetErrorString(e));
     return NM_OK;
 }
 

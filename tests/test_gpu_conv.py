@@ -23,13 +23,25 @@ def _plans(nm, s):
         p = nm.nm_plan_t()
         p.variant, p.split = variant, split
         out.append(p)
+    # stream kernel: default width, 256 channels per CTA (one accumulator buffer), one tile per CTA,
+    # and a two-stage ring (every stage reused many times)
+    for bn, stages in ((0, 0), (256, 0), (s.tile_t if s is not None else 16, 0), (0, 2)):
+        p = nm.nm_plan_t()
+        p.variant, p.bn, p.stages = 3, bn, stages
+        out.append(p)
+    # expanded-operand kernel: default width, 32 and 256 channels per work item, two-stage ring
+    for bn, stages in ((0, 0), (32, 0), (256, 0), (0, 2)):
+        p = nm.nm_plan_t()
+        p.variant, p.bn, p.stages = 4, bn, stages
+        out.append(p)
     return out
 
 
-def _run(nm, s, integer=False, use_bias=True):
+def _run(nm, s, integer=False, use_bias=True, need_variant=None):
     w, x, b = tensors_for(s, integer)
     vr, ir, yr = oracle_layer(s, w, x, b, use_bias)
     ran = 0
+    variants_run = set()
     for plan in _plans(nm, s):
         try:
             _, v, i, y = gpu_layer(nm, s, w, x, b, use_bias, plan)
@@ -38,6 +50,7 @@ def _run(nm, s, integer=False, use_bias=True):
                 continue  # this variant does not take the shape
             raise
         ran += 1
+        variants_run.add(plan.variant if plan is not None else 0)
         assert_prune_bit_exact(v, i, vr, ir)
         if integer:
             # every product and partial sum is exact in TF32 / fp32: results must be identical
@@ -45,6 +58,8 @@ def _run(nm, s, integer=False, use_bias=True):
         else:
             assert_conv_close(y, yr)
     assert ran >= 2  # the default and at least one explicit variant
+    for v in need_variant or ():
+        assert v in variants_run, f"variant {v} did not take {s.name}"
 
 
 def test_tiny_config(nm):
@@ -83,7 +98,7 @@ def test_small_shapes(nm, s):
 # inputs of at least 128 KiB with c_in % 32 == 0: these take the TMA (im2col) producer
 MEDIUM = [
     ConvShape("tma_3x3", 2, 16, 16, 64, 64, 3, 3, 1, 1, 1, 2, 4, 32),
-    ConvShape("tma_ragged_tail", 3, 13, 13, 64, 64, 3, 3, 1, 1, 1, 2, 4, 64),      # 507 pixels
+    ConvShape("tma_ragged_tail", 3, 13, 13, 96, 64, 3, 3, 1, 1, 1, 2, 4, 64),      # 507 pixels
     ConvShape("tma_stride2", 2, 15, 15, 128, 64, 3, 3, 2, 1, 1, 2, 4, 32),
     ConvShape("tma_dilation2", 1, 20, 20, 96, 32, 3, 3, 1, 2, 2, 2, 4, 32),
     ConvShape("tma_1x1", 2, 14, 14, 256, 96, 1, 1, 1, 0, 1, 2, 4, 32),
@@ -94,15 +109,30 @@ MEDIUM = [
     ConvShape("tma_3of4", 1, 16, 16, 128, 64, 1, 1, 1, 0, 1, 3, 4, 64),
     ConvShape("tma_dense", 1, 16, 16, 128, 48, 3, 3, 1, 1, 1, 4, 4, 16),
     ConvShape("tma_tile128", 1, 16, 16, 128, 256, 3, 3, 1, 1, 1, 2, 4, 128),
+    ConvShape("tma_dense_64", 1, 16, 16, 128, 64, 3, 3, 1, 1, 1, 4, 4, 32),
+    ConvShape("tma_tile256", 1, 16, 16, 128, 512, 1, 1, 1, 0, 1, 2, 4, 256),
+    ConvShape("tma_1of4", 2, 15, 15, 96, 128, 3, 3, 1, 1, 1, 1, 4, 64),
+    ConvShape("tma_2of8", 2, 15, 15, 128, 128, 3, 3, 1, 1, 1, 2, 8, 32),
+    ConvShape("tma_4of8", 1, 20, 20, 128, 64, 1, 1, 1, 0, 1, 4, 8, 16),
+    ConvShape("tma_cin32_3x3", 2, 20, 20, 32, 64, 3, 3, 1, 1, 1, 2, 4, 16),          # K = 288: half-filled last chunk
+    ConvShape("tma_many_items", 8, 56, 56, 32, 128, 1, 1, 1, 0, 1, 2, 4, 64),        # 196 work items: several per CTA
+    ConvShape("tma_many_items_3x3", 4, 56, 56, 32, 64, 3, 3, 1, 1, 1, 2, 4, 32),     # 196 work items of 5 chunks, last chunk half-filled
+    ConvShape("tma_wide_256", 2, 28, 28, 64, 512, 1, 1, 1, 0, 1, 2, 4, 64),          # 4 tiles per CTA at bn = 256
 ]
 
 
 @pytest.mark.parametrize("s", MEDIUM, ids=lambda s: s.name)
 def test_medium_shapes(nm, s):
-    _run(nm, s)
+    # the stream kernel takes tiles that are multiples of 16 channels and its seven N:M patterns
+    # on inputs of at least 128 KiB
+    stream = (s.tile_t % 16 == 0 and s.c_out % 32 == 0 and s.batch * s.h * s.w * s.c_in * 4 >= 131072 and
+              (s.n_keep, s.m_group) in ((1, 4), (2, 4), (3, 4), (4, 4), (1, 8), (2, 8), (4, 8)))
+    big = s.batch * s.h * s.w * s.c_in * 4 >= 131072
+    expand = big and s.c_in % 32 == 0 and s.c_out % 32 == 0     # any tile width, any N:M
+    _run(nm, s, need_variant=[3 if stream else 2] + ([4] if expand else []))
 
 
-@pytest.mark.parametrize("s", MEDIUM[:6], ids=lambda s: s.name)
+@pytest.mark.parametrize("s", MEDIUM[:6] + MEDIUM[13:], ids=lambda s: s.name)
 def test_medium_shapes_integer_exact(nm, s):
     _run(nm, s, integer=True)
 
@@ -119,7 +149,12 @@ def test_asymmetric_geometry(nm):
     yr = oracle.conv2d(vr, ir, 3, 5, 64, 16, x.numpy(), stride, pad, dil, b.numpy(), True)
     hnd = nm.nm_prune(w.cuda(), 2, 4, 16)
     for plan in _plans(nm, None):
-        y = nm.nm_conv2d(hnd, x.cuda(), 3, 5, stride, pad, dil, b.cuda(), True, plan=plan)
+        try:
+            y = nm.nm_conv2d(hnd, x.cuda(), 3, 5, stride, pad, dil, b.cuda(), True, plan=plan)
+        except nm.NmError as e:
+            if plan is not None and e.status == nm.NM_ERR_UNSUPPORTED:
+                continue
+            raise
         nm.nm_weights_check(hnd)
         torch.cuda.synchronize()
         assert np.array_equal(y.cpu().numpy(), yr), f"plan {plan.as_dict() if plan else None}"
