@@ -12,7 +12,8 @@
 // bound by HBM and the tensor pipe has slack; the auto-tuner decides per layer by measurement.
 // The pruning tile width plays no role here, so any tile_t is accepted.
 //
-//   producer (1 thread)   TMA im2col load of the slab + tiled load of the weight block per stage
+//   producer (1 thread)   TMA im2col load of the slab + one contiguous bulk copy of the weight block
+//                         (stored pre-swizzled, so it costs no per-row TMA requests) per stage
 //   MMA issuer (1 thread) four 128 x BN x 8 TF32 tcgen05.mma (SS) per stage into one of two
 //                         accumulator buffers in tensor memory
 //   epilogue (8 warps)    TMEM -> registers, + bias, ReLU, swizzled staging, TMA store to NHWC;
@@ -47,7 +48,7 @@ __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0;
 
 __global__ void __launch_bounds__(THREADS, 1)
 k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ CUtensorMap tm_x,
-              const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y)
+              const __grid_constant__ CUtensorMap tm_y)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[NSTAGE_MAX], s_free[NSTAGE_MAX], s_accfull[2], s_accfree[2];
@@ -73,7 +74,6 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         mbar_fence_init();
         s_abort = 0;
         tma_prefetch_desc(&tm_x);
-        tma_prefetch_desc(&tm_w);
         tma_prefetch_desc(&tm_y);
     }
     tc_fence_before();
@@ -84,9 +84,12 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     if (warp == 0) {
         // =========================== producer ===========================
         if (lane == 0) {
+            int issued = 0;
             const int hw = p.ho * p.wo;
             const uint32_t tx = SUB_BYTES + static_cast<uint32_t>(cfg.bn) * 128u;
-            long long cc = 0;
+            const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
+            const size_t w_step = static_cast<size_t>(p.c_out) * 32;   // floats between two 32-column blocks
+            RingPos rp;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
                 const int slice = static_cast<int>(work % cfg.n_slices);
                 const long long pix0 = (work / cfg.n_slices) * BM;
@@ -94,26 +97,34 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 const int rem = static_cast<int>(pix0 - static_cast<long long>(n0) * hw);
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
-                int tap = 0, ch = 0;
-                for (int c = 0; c < n_sub; ++c, ++cc) {
-                    const int s = static_cast<int>(cc % NS);
-                    if (cc >= NS && !mbar_wait(smem_u32(&s_free[s]), static_cast<uint32_t>((cc / NS) - 1) & 1u))
-                        *abort_flag = 2;
+                const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32;
+                int ch = 0, off_w = 0, off_h = 0, tw = 0;
+                for (int c = 0; c < n_sub; ++c) {
+                    if (rp.wrapped && !mbar_wait(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
-                    const uint32_t a_smem = ring + s * cfg.stage_bytes;
-                    const uint32_t bar = smem_u32(&s_full[s]);
+                    const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
+                    const uint32_t bar = smem_u32(&s_full[rp.s]);
                     mbar_arrive_expect_tx(bar, tx);
-                    tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>((tap % p.kw) * p.dil_w),
-                                       static_cast<uint16_t>((tap / p.kw) * p.dil_h));
-                    tma_load_2d(a_smem + SUB_BYTES, &tm_w, bar, c * 32, slice * cfg.bn);
+                    tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>(off_w),
+                                       static_cast<uint16_t>(off_h));
+                    bulk_load_1d(a_smem + SUB_BYTES, wsrc, w_bytes, bar);
+                    wsrc += w_step;
                     ch += 32;
-                    if (ch >= p.c_in) { ch = 0; ++tap; }
+                    if (ch >= p.c_in) {
+                        ch = 0;
+                        off_w += p.dil_w;
+                        if (++tw == p.kw) { tw = 0; off_w = 0; off_h += p.dil_h; }
+                    }
+                    rp.advance(NS);
+                    ++issued;
                 }
             }
             if (aborted(abort_flag)) {
-                for (long long back = 1; back <= NS && back <= cc; ++back) {
-                    const long long cl = cc - back;
-                    (void)mbar_wait(smem_u32(&s_full[cl % NS]), static_cast<uint32_t>(cl / NS) & 1u);
+                // loads already issued still target this CTA's shared memory: let them land
+                for (int back = 0; back < NS && back < issued; ++back) {
+                    if (rp.s == 0) { rp.s = NS; rp.parity ^= 1u; }
+                    --rp.s;
+                    (void)mbar_wait(smem_u32(&s_full[rp.s]), rp.parity);
                 }
             }
         }
@@ -121,29 +132,32 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
-            long long cc = 0, ti = 0;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x, ++ti) {
-                const int ab = static_cast<int>(ti & 1);
-                if (ti >= 2 && !mbar_wait(smem_u32(&s_accfree[ab]), static_cast<uint32_t>((ti >> 1) - 1) & 1u)) {
+            RingPos rp;
+            uint32_t ab = 0, acc_par = 0;   // accumulator buffer of this item, parity of its current use
+            bool acc_wrapped = false;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+                if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
                     *abort_flag = 5;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
-                for (int c = 0; c < n_sub; ++c, ++cc) {
-                    const int s = static_cast<int>(cc % NS);
-                    if (!mbar_wait(smem_u32(&s_full[s]), static_cast<uint32_t>(cc / NS) & 1u)) { *abort_flag = 6; break; }
+                for (int c = 0; c < n_sub; ++c) {
+                    if (!mbar_wait(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     tc_fence_after();
-                    const uint32_t a_smem = ring + s * cfg.stage_bytes;
+                    const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     const uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
                     const uint64_t bdesc = umma_desc_k_sw128(a_smem + SUB_BYTES, 1024);
 #pragma unroll
                     for (int kq = 0; kq < 4; ++kq)
                         umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > 0 || kq > 0) ? 1u : 0u);
-                    umma_commit(smem_u32(&s_free[s]));
+                    umma_commit(smem_u32(&s_free[rp.s]));
+                    rp.advance(NS);
                 }
                 if (aborted(abort_flag)) break;
                 umma_commit(smem_u32(&s_accfull[ab]));
+                if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
+                ab ^= 1u;
             }
         }
     } else if (warp >= 4) {
@@ -154,13 +168,12 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         const uint32_t my_staging = staging + (warp - 4) * 2 * 4096;
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
-        long long ti = 0;
-        uint32_t nb = 0;
+        uint32_t nb = 0, ti = 0;
         for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
             const int slice = static_cast<int>(work % cfg.n_slices);
             const long long pix0 = (work / cfg.n_slices) * BM;
-            const int ab = static_cast<int>(ti & 1);
-            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), static_cast<uint32_t>(ti >> 1) & 1u);
+            const int ab = static_cast<int>(ti & 1u);
+            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
@@ -269,18 +282,6 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     return true;
 }
 
-// Dense [c_out][K] weights as a tiled map with a 32-column x `rows` box.
-bool encode_wx(const ConvParams& p, int rows, CUtensorMap* tm)
-{
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.k), static_cast<cuuint64_t>(p.c_out)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(p.k) * 4};
-    const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(rows)};
-    const cuuint32_t es[2] = {1, 1};
-    return nmtm::encoders().tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(p.wx), dims, strides, box,
-                                  es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 namespace nmhost {
@@ -296,15 +297,15 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     ExpandCfg cfg;
     if (!make_cfg(p, plan, &cfg))
         return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the expanded-operand kernel does not take this layer / plan");
-    alignas(64) CUtensorMap tm_x, tm_w, tm_y;
-    if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !encode_wx(p, cfg.bn, &tm_w) || !nmtm::encode_y_tiled(p, &tm_y))
+    alignas(64) CUtensorMap tm_x, tm_y;
+    if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_y_tiled(p, &tm_y))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 4)");
     size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + STAGING_BYTES;
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
     cudaError_t e = cudaFuncSetAttribute(k_conv_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    k_conv_expand<<<static_cast<unsigned>(grid), THREADS, smem, st>>>(p, cfg, tm_x, tm_w, tm_y);
+    k_conv_expand<<<static_cast<unsigned>(grid), THREADS, smem, st>>>(p, cfg, tm_x, tm_y);
     count_launch(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 4): %s", cudaGetErrorString(e));

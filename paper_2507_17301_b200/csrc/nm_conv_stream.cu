@@ -163,7 +163,8 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
             const int hw = p.ho * p.wo;
             const size_t rpitch = static_cast<size_t>(n_chunks) * 32;
             const uint32_t tx_fixed = static_cast<uint32_t>(cfg.bn) * 128u + static_cast<uint32_t>(g) * 32u;
-            long long cc = 0;
+            RingPos rp;
+            int issued = 0;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
                 const int slice = static_cast<int>(work % cfg.n_slices);
                 const long long pix0 = (work / cfg.n_slices) * BM;
@@ -171,36 +172,41 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                 const int rem = static_cast<int>(pix0 - static_cast<long long>(n0) * hw);
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
-                for (int c = 0; c < n_chunks; ++c, ++cc) {
-                    const int s = static_cast<int>(cc % NS);
-                    if (cc >= NS && !mbar_wait(smem_u32(&s_free[s]), static_cast<uint32_t>((cc / NS) - 1) & 1u))
-                        *abort_flag = 2;
+                const uint8_t* rsrc = p.rel2 + static_cast<size_t>(slice * g) * rpitch;
+                int ch = 0, off_w = 0, off_h = 0, tw = 0, k0 = 0;   // position of the next 32-column sub-tile
+                for (int c = 0; c < n_chunks; ++c) {
+                    if (rp.wrapped && !mbar_wait(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
-                    const uint32_t b_smem = ring + s * cfg.stage_bytes;
+                    const uint32_t b_smem = ring + rp.s * cfg.stage_bytes;
                     const uint32_t slab = b_smem + cfg.b_bytes;
                     const uint32_t relbuf = slab + P::SEGS * SUB_BYTES;
-                    const uint32_t bar = smem_u32(&s_full[s]);
-                    int live = 0;
-                    for (int seg = 0; seg < P::SEGS; ++seg) live += (c * P::S + seg * 32 < p.k) ? 1 : 0;
+                    const uint32_t bar = smem_u32(&s_full[rp.s]);
+                    const int live = (P::SEGS == 2 && k0 + 32 >= p.k) ? 1 : P::SEGS;
                     mbar_arrive_expect_tx(bar, static_cast<uint32_t>(live) * SUB_BYTES + tx_fixed);
-                    for (int seg = 0; seg < live; ++seg) {
-                        const int k0 = c * P::S + seg * 32;
-                        const int tap = k0 / p.c_in, ch = k0 - tap * p.c_in;
-                        tma_load_im2col_4d(slab + seg * SUB_BYTES, &tm_x, bar, ch, w0, h0, n0,
-                                           static_cast<uint16_t>((tap % p.kw) * p.dil_w),
-                                           static_cast<uint16_t>((tap / p.kw) * p.dil_h));
+                    for (int seg = 0; seg < P::SEGS; ++seg) {
+                        if (seg < live)
+                            tma_load_im2col_4d(slab + seg * SUB_BYTES, &tm_x, bar, ch, w0, h0, n0,
+                                               static_cast<uint16_t>(off_w), static_cast<uint16_t>(off_h));
+                        k0 += 32;
+                        ch += 32;
+                        if (ch >= p.c_in) {
+                            ch = 0;
+                            off_w += p.dil_w;
+                            if (++tw == p.kw) { tw = 0; off_w = 0; off_h += p.dil_h; }
+                        }
                     }
                     tma_load_2d(b_smem, &tm_w, bar, c * 32, slice * cfg.bn);
-                    for (int t = 0; t < g; ++t)
-                        bulk_load_1d(relbuf + t * 32, p.rel2 + static_cast<size_t>(slice * g + t) * rpitch + c * 32, 32u,
-                                     bar);
+                    for (int t = 0; t < g; ++t) bulk_load_1d(relbuf + t * 32, rsrc + t * rpitch + c * 32, 32u, bar);
+                    rp.advance(NS);
+                    ++issued;
                 }
             }
             if (aborted(abort_flag)) {
                 // loads already issued still target this CTA's shared memory: let them land
-                for (long long back = 1; back <= NS && back <= cc; ++back) {
-                    const long long cl = cc - back;
-                    (void)mbar_wait(smem_u32(&s_full[cl % NS]), static_cast<uint32_t>(cl / NS) & 1u);
+                for (int back = 0; back < NS && back < issued; ++back) {
+                    if (rp.s == 0) { rp.s = NS; rp.parity ^= 1u; }
+                    --rp.s;
+                    (void)mbar_wait(smem_u32(&s_full[rp.s]), rp.parity);
                 }
             }
         }
@@ -208,23 +214,23 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(BM, T);
-            long long cc = 0, ti = 0;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x, ++ti) {
-                const int ab = static_cast<int>(ti % cfg.n_acc);
-                if (ti >= cfg.n_acc &&
-                    !mbar_wait(smem_u32(&s_accfree[ab]), static_cast<uint32_t>((ti / cfg.n_acc) - 1) & 1u)) {
+            RingPos rp;
+            uint32_t set = 0, set_par = 0;          // operand set of this chunk, parity of its current use
+            uint32_t ab = 0, acc_par = 0;           // accumulator buffer of this item, parity of its current use
+            bool acc_wrapped = false;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+                if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
                     *abort_flag = 5;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
-                for (int c = 0; c < n_chunks; ++c, ++cc) {
-                    const int s = static_cast<int>(cc % NS), set = static_cast<int>(cc & 1);
-                    if (!mbar_wait(smem_u32(&s_full[s]), static_cast<uint32_t>(cc / NS) & 1u)) { *abort_flag = 6; break; }
-                    if (!mbar_wait(smem_u32(&s_aready[set]), static_cast<uint32_t>(cc >> 1) & 1u)) { *abort_flag = 7; break; }
+                for (int c = 0; c < n_chunks; ++c) {
+                    if (!mbar_wait(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
+                    if (!mbar_wait(smem_u32(&s_aready[set]), set_par)) { *abort_flag = 7; break; }
                     if (aborted(abort_flag)) break;
                     tc_fence_after();
-                    const uint32_t b_smem = ring + s * cfg.stage_bytes;
+                    const uint32_t b_smem = ring + rp.s * cfg.stage_bytes;
                     const uint32_t a_set = tmem + A_COL0 + set * cfg.set_cols;
                     for (int t = 0; t < g; ++t) {
                         const uint64_t bdesc = umma_desc_k_sw128(b_smem + t * T * 128, 1024);
@@ -234,10 +240,20 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                                          (c > 0 || kq > 0) ? 1u : 0u);
                     }
                     umma_commit(smem_u32(&s_afree[set]));
-                    umma_commit(smem_u32(&s_free[s]));
+                    umma_commit(smem_u32(&s_free[rp.s]));
+                    rp.advance(NS);
+                    if (set == 1) set_par ^= 1u;
+                    set ^= 1u;
                 }
                 if (aborted(abort_flag)) break;
                 umma_commit(smem_u32(&s_accfull[ab]));
+                if (cfg.n_acc == 2) {
+                    if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
+                    ab ^= 1u;
+                } else {
+                    acc_par ^= 1u;
+                    acc_wrapped = true;
+                }
             }
         }
     } else if (warp >= 4 && warp < 8) {
@@ -247,14 +263,14 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
         const uint32_t my_staging = staging + q * 2 * 4096;
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
-        long long ti = 0;
+        uint32_t ti = 0;
         uint32_t nb = 0;  // staging boxes this warp has filled so far
         for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
             const int slice = static_cast<int>(work % cfg.n_slices);
             const long long pix0 = (work / cfg.n_slices) * BM;
-            const int ab = static_cast<int>(ti % cfg.n_acc);
+            const int ab = cfg.n_acc == 2 ? static_cast<int>(ti & 1u) : 0;
             const bool ok = aborted(abort_flag) ||
-                            mbar_wait(smem_u32(&s_accfull[ab]), static_cast<uint32_t>(ti / cfg.n_acc) & 1u);
+                            mbar_wait(smem_u32(&s_accfull[ab]), (cfg.n_acc == 2 ? (ti >> 1) : ti) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
@@ -308,13 +324,15 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t rx = static_cast<uint32_t>(row & 7);
         constexpr int CI0_STEP = P::LW;   // first 16-byte piece of half `wg`
-        long long cc = 0;
+        RingPos rp;
+        uint32_t set = 0, set_par = 0;
+        bool set_wrapped = false;
         for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-            for (int c = 0; c < n_chunks; ++c, ++cc) {
-                const int s = static_cast<int>(cc % NS), set = static_cast<int>(cc & 1);
-                bool ok = mbar_wait(smem_u32(&s_full[s]), static_cast<uint32_t>(cc / NS) & 1u);
+            for (int c = 0; c < n_chunks; ++c) {
+                const int s = rp.s;
+                bool ok = mbar_wait(smem_u32(&s_full[s]), rp.parity);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 3;
-                ok = cc < 2 || mbar_wait(smem_u32(&s_afree[set]), static_cast<uint32_t>((cc >> 1) - 1) & 1u);
+                ok = !set_wrapped || mbar_wait(smem_u32(&s_afree[set]), set_par ^ 1u);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
                 if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
                 tc_fence_after();
@@ -358,6 +376,9 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                     mbar_arrive(smem_u32(&s_aready[set]));
                     mbar_arrive(smem_u32(&s_free[s]));
                 }
+                rp.advance(NS);
+                if (set == 1) { set_par ^= 1u; set_wrapped = true; }
+                set ^= 1u;
             }
         }
     }

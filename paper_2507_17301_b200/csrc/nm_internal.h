@@ -28,7 +28,7 @@ struct nm_weights {
     float* wt2;          // [c_out][v2_chunks * 32] TF32 weights, chunk-major, first v2_kc of each 32 used
     uint8_t* rel2;       // [n_tiles][v2_chunks * 32] source column of each kept column, relative to its chunk
     // Expanded layout (variant 4): the pruned matrix back in dense shape, zeros in the pruned columns.
-    float* wx;           // [c_out][k] TF32, or NULL when the layer shape rules the variant out
+    float* wx;           // [k / 32][c_out][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
 };
 
 // Geometry handed to the convolution kernels.

@@ -120,15 +120,20 @@ __global__ void k_build_slab(const float* __restrict__ values, const uint16_t* _
     if (o == r * tile_t) rel2[static_cast<size_t>(r) * pitch + chunk * 32 + jj] = static_cast<uint8_t>(col - chunk * s_cols);
 }
 
-// Expanded layout: wx[o][indices[o / T][j]] = TF32(values[o][j]); the rest stays zero.
-__global__ void k_expand(const float* __restrict__ values, const uint16_t* __restrict__ indices, int k, int kk,
+// Expanded layout: element (o, k) = TF32(values[o][j]) where k = indices[o / T][j], zero elsewhere,
+// stored as the shared-memory image the tensor core reads: blocks of 32 columns, inside a block
+// one 128-byte row per output channel whose 16-byte pieces are XOR-ed with (o % 8) (the 128-byte
+// swizzle), so that any run of channels starting at a multiple of 8 is one contiguous bulk copy.
+__global__ void k_expand(const float* __restrict__ values, const uint16_t* __restrict__ indices, int c_out, int kk,
                          int tile_t, float* __restrict__ wx)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     const int o = blockIdx.y;
     if (j >= kk) return;
     const int col = indices[static_cast<size_t>(o / tile_t) * kk + j];
-    wx[static_cast<size_t>(o) * k + col] = nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
+    const int blk = col >> 5, kc = col & 31;
+    wx[(static_cast<size_t>(blk) * c_out + o) * 32 + ((((kc >> 2) ^ (o & 7)) << 2) | (kc & 3))] =
+        nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
 }
 
 // Import path: every index row must be strictly ascending and below k.
@@ -231,7 +236,7 @@ nm_status_t build_expanded_layout(nm_weights* h, cudaStream_t st)
     cudaError_t e = cudaMemsetAsync(h->wx, 0, bytes, st);
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "expanded layout memset: %s", cudaGetErrorString(e));
     const dim3 grid((h->kk + 127) / 128, h->c_out);
-    k_expand<<<grid, 128, 0, st>>>(h->values, h->indices, h->k, h->kk, h->tile_t, h->wx);
+    k_expand<<<grid, 128, 0, st>>>(h->values, h->indices, h->c_out, h->kk, h->tile_t, h->wx);
     count_launch(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "expanded layout kernel: %s", cudaGetErrorString(e));

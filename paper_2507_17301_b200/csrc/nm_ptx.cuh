@@ -58,6 +58,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     return false;
 }
 
+// Position in a ring of `n` mbarrier-guarded stages: stage index and the parity of its current
+// use, advanced without divisions (a lone producer or issuer thread runs at one dependent
+// instruction every few cycles, so a 64-bit modulo per stage would dominate its loop).
+struct RingPos {
+    int s = 0;
+    uint32_t parity = 0;
+    bool wrapped = false;   // every stage has been used at least once
+    __device__ __forceinline__ void advance(int n)
+    {
+        if (++s == n) {
+            s = 0;
+            parity ^= 1u;
+            wrapped = true;
+        }
+    }
+};
+
 // ---- cp.async -----------------------------------------------------------------------------------
 // 16-byte copy; src_bytes = 0 writes zeros (used for padding taps and rows past the end).
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
