@@ -129,6 +129,7 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
     switch (variant) {
         case 0:
             if (nmhost::stream_plan_ok(p, nullptr)) return nmhost::launch_conv_stream(p, nullptr, st);
+            if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, nullptr)) return nmhost::launch_conv_rowrun(p, nullptr, st);
             if (nmhost::slab_plan_ok(p, nullptr)) return nmhost::launch_conv_slab(p, nullptr, st);
             return nmhost::launch_conv_gather(p, st);
         case 1:
@@ -139,6 +140,8 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
             return nmhost::launch_conv_stream(p, plan, st);
         case 4:
             return nmhost::launch_conv_expand(p, plan, st);
+        case 5:
+            return nmhost::launch_conv_rowrun(p, plan, st);
         default:
             return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
     }
@@ -149,6 +152,9 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
 {
     std::vector<nm_plan_t> out;
     nm_plan_t a;
+    std::memset(&a, 0, sizeof(a));
+    a.variant = 5;                          // row-run kernel (few input channels)
+    if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, &a)) out.push_back(a);
     std::memset(&a, 0, sizeof(a));
     for (int bn : {64, 128, 256}) {         // expanded-operand kernel
         a.variant = 4; a.bn = bn; a.stages = 0;

@@ -28,7 +28,7 @@ struct nm_weights {
     float* wt2;          // [c_out][v2_chunks * 32] TF32 weights, chunk-major, first v2_kc of each 32 used
     uint8_t* rel2;       // [n_tiles][v2_chunks * 32] source column of each kept column, relative to its chunk
     // Expanded layout (variant 4): the pruned matrix back in dense shape, zeros in the pruned columns.
-    float* wx;           // [k / 32][c_out][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
+    float* wx;           // [ceil(k / 32)][c_out][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
 };
 
 // Geometry handed to the convolution kernels.
@@ -76,6 +76,10 @@ nm_status_t launch_conv_slab(const ConvParams& p, const nm_plan_t* plan, cudaStr
 // nm_conv_expand.cu — variant 4
 bool expand_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
+// nm_conv_rowrun.cu — variant 5
+bool rowrun_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_rowrun(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 
 // nm_conv_stream.cu — variant 3
 bool stream_plan_ok(const ConvParams& p, const nm_plan_t* plan);

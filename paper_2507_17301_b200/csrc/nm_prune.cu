@@ -225,9 +225,10 @@ nm_status_t build_slab_layout(nm_weights* h, cudaStream_t st)
 nm_status_t build_expanded_layout(nm_weights* h, cudaStream_t st)
 {
     h->wx = nullptr;
-    // only shapes the expanded-operand kernel takes: whole 32-column slabs, 32-channel output blocks
-    if (h->c_in % 32 != 0 || h->c_out % 32 != 0 || h->kk == 0) return NM_OK;
-    const size_t bytes = static_cast<size_t>(h->c_out) * h->k * sizeof(float);
+    // only shapes the kernels that read it take: 32-channel output blocks, and either whole
+    // 32-column slabs (expanded-operand kernel) or a short reduction axis (row-run kernel)
+    if (h->c_out % 32 != 0 || h->kk == 0 || (h->c_in % 32 != 0 && h->k > 512)) return NM_OK;
+    const size_t bytes = static_cast<size_t>((h->k + 31) / 32) * h->c_out * 32 * sizeof(float);
     if (cudaMalloc(&h->wx, bytes) != cudaSuccess) {
         (void)cudaGetLastError();
         h->wx = nullptr;

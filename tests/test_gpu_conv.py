@@ -34,6 +34,9 @@ def _plans(nm, s):
         p = nm.nm_plan_t()
         p.variant, p.bn, p.stages = 4, bn, stages
         out.append(p)
+    p = nm.nm_plan_t()
+    p.variant = 5                                     # row-run kernel
+    out.append(p)
     return out
 
 
@@ -119,6 +122,28 @@ MEDIUM = [
     ConvShape("tma_many_items_3x3", 4, 56, 56, 32, 64, 3, 3, 1, 1, 1, 2, 4, 32),     # 196 work items of 5 chunks, last chunk half-filled
     ConvShape("tma_wide_256", 2, 28, 28, 64, 512, 1, 1, 1, 0, 1, 2, 4, 64),          # 4 tiles per CTA at bn = 256
 ]
+
+
+# few input channels, c_out a multiple of 32, dil_w = 1, output rows of at most 128 pixels: row-run kernel
+ROWRUN = [
+    ConvShape("rr_stem", 2, 64, 64, 3, 64, 7, 7, 2, 3, 1, 1, 1, 64),
+    ConvShape("rr_stem_wide", 1, 40, 252, 3, 32, 7, 7, 2, 3, 1, 1, 1, 32),          # 126 output pixels per row
+    ConvShape("rr_3x3_c4", 2, 20, 20, 4, 64, 3, 3, 1, 1, 1, 2, 4, 8),                # pruned, tile 8
+    ConvShape("rr_5x5_c8_s1", 1, 30, 30, 8, 64, 5, 5, 1, 2, 1, 2, 4, 32),
+    ConvShape("rr_nopad", 1, 24, 24, 4, 32, 3, 3, 1, 0, 1, 4, 4, 32),
+    ConvShape("rr_1x1_c12", 3, 10, 16, 12, 128, 1, 1, 1, 0, 1, 1, 4, 16),
+    ConvShape("rr_k500", 2, 12, 12, 20, 32, 5, 5, 2, 2, 1, 2, 4, 32),                # K = 500: 16 sub-tiles
+]
+
+
+@pytest.mark.parametrize("s", ROWRUN, ids=lambda s: s.name)
+def test_rowrun_shapes(nm, s):
+    _run(nm, s, need_variant=[5])
+
+
+@pytest.mark.parametrize("s", ROWRUN[:4], ids=lambda s: s.name)
+def test_rowrun_shapes_integer_exact(nm, s):
+    _run(nm, s, integer=True, need_variant=[5])
 
 
 @pytest.mark.parametrize("s", MEDIUM, ids=lambda s: s.name)
