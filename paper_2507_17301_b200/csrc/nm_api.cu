@@ -189,6 +189,14 @@ nm_status_t fail(nm_status_t s, const char* fmt, ...)
     va_end(ap);
     return s;
 }
+bool pdl_enabled()
+{
+    static const bool on = [] {
+        const char* v = std::getenv("NM_NO_PDL");
+        return !(v && v[0] == '1');
+    }();
+    return on;
+}
 void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
 }  // namespace nmhost
 

@@ -32,7 +32,7 @@ constexpr int BM = 128;
 constexpr int SUB_BYTES = BM * 128;
 constexpr int NSTAGE_MAX = 8;
 constexpr int THREADS = 384;                   // 4 service warps + 8 epilogue warps
-constexpr int STAGING_BYTES = 8 * 2 * 4096;    // per epilogue warp two 32 x 32 output boxes
+constexpr int BOX_BYTES = 4096;                // one 32-pixel x 32-channel output box
 
 struct ExpandCfg {
     int bn;           // output channels per work item
@@ -41,6 +41,7 @@ struct ExpandCfg {
     int b_bytes;      // weight bytes per stage (bn rows of 128 bytes)
     int stage_bytes;
     int n_sub;        // K / 32
+    int boxes;        // output staging boxes per epilogue warp: 2 for short reductions, 1 when the ring needs the room
     long long n_work;
 };
 
@@ -80,6 +81,8 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
+    pdl_launch_dependents();   // the next kernel may start its own set-up as SMs become free
+    pdl_wait();                // from here on global memory written by the previous kernel is read
 
     if (warp == 0) {
         // =========================== producer ===========================
@@ -165,7 +168,8 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         const int q = warp & 3;            // TMEM lane quadrant
         const int half = (warp - 4) >> 2;  // which channel blocks of 32: blk = 2 * i + half
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const uint32_t my_staging = staging + (warp - 4) * 2 * 4096;
+        const uint32_t my_staging = staging + (warp - 4) * cfg.boxes * BOX_BYTES;
+        const uint32_t box_toggle = cfg.boxes == 2 ? 1u : 0u;
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t nb = 0, ti = 0;
@@ -187,8 +191,12 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
                 }
-                const uint32_t box = my_staging + (nb & 1u) * 4096;
-                if (lane == 0 && nb >= 2) tma_store_wait_read_n<1>();
+                const uint32_t box = my_staging + (nb & box_toggle) * BOX_BYTES;
+                if (lane == 0) {
+                    // the store that last read this box must be done with it
+                    if (cfg.boxes == 2) { if (nb >= 2) tma_store_wait_read_n<1>(); }
+                    else if (nb >= 1) tma_store_wait_read_n<0>();
+                }
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
 #pragma unroll
@@ -268,7 +276,8 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     cfg->b_bytes = ((bn * 128 + 1023) / 1024) * 1024;
     cfg->stage_bytes = SUB_BYTES + cfg->b_bytes;
     cfg->n_sub = p.k / 32;
-    const int budget = 227 * 1024 - 1024 - STAGING_BYTES - 1024;
+    cfg->boxes = cfg->n_sub <= 8 ? 2 : 1;   // long reductions: the epilogue is rare, the ring needs the bytes
+    const int budget = 227 * 1024 - 1024 - 8 * cfg->boxes * BOX_BYTES - 1024;
     int stages = plan && plan->stages > 0 ? plan->stages : NSTAGE_MAX;
     if (stages > NSTAGE_MAX) return false;
     if (plan && plan->stages > 0) {
@@ -300,14 +309,14 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     alignas(64) CUtensorMap tm_x, tm_y;
     if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_y_tiled(p, &tm_y))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 4)");
-    size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + STAGING_BYTES;
+    size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 8 * cfg.boxes * BOX_BYTES;
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
     cudaError_t e = cudaFuncSetAttribute(k_conv_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    k_conv_expand<<<static_cast<unsigned>(grid), THREADS, smem, st>>>(p, cfg, tm_x, tm_y);
-    count_launch(1);
-    e = cudaGetLastError();
+    e = nmhost::launch_pdl(k_conv_expand, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x, tm_y);
+    nmhost::count_launch(1);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 4): %s", cudaGetErrorString(e));
     return NM_OK;
 }

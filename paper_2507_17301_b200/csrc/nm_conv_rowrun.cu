@@ -99,6 +99,8 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
+    pdl_launch_dependents();   // the next kernel may start its own set-up as SMs become free
+    pdl_wait();                // from here on global memory written by the previous kernel is read
 
     if (warp == 0) {
         // =========================== producer ===========================
@@ -249,15 +251,22 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                         step = p.stride_w * p.c_in * 4;
                     }
                 }
-                const uint32_t dst0 = a_ring + rp.s * SUB_BYTES + ((lane & 3) << 2);
-                const uint32_t c16 = static_cast<uint32_t>(lane >> 2);
-#pragma unroll 4
+                // rows bw, bw + 8, ...: (row % 8) is the same for all of them, so is the swizzle term
+                uint32_t dst = a_ring + rp.s * SUB_BYTES + ((lane & 3) << 2) + bw * 128 +
+                               ((static_cast<uint32_t>(lane >> 2) ^ static_cast<uint32_t>(bw)) << 4);
+                src += bw * step;
+                const int step8 = step * 8;
+                uint32_t v[BM / 8];
+#pragma unroll
                 for (int i = 0; i < BM / 8; ++i) {
-                    const int row = bw + i * 8;
-                    uint32_t v;
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(row < p.wo ? src + row * step : zero_row));
-                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(dst0 + row * 128 + ((c16 ^ (row & 7)) << 4)), "r"(v)
-                                 : "memory");
+                    // tile rows past the end of the output row read the row of zeros
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(bw + i * 8 < p.wo ? src : zero_row));
+                    src += step8;
+                }
+#pragma unroll
+                for (int i = 0; i < BM / 8; ++i) {
+                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(dst), "r"(v[i]) : "memory");
+                    dst += 8 * 128;
                 }
                 fence_proxy_async();
                 __syncwarp();
@@ -362,9 +371,9 @@ nm_status_t launch_conv_rowrun(const ConvParams& p, const nm_plan_t* /*plan*/, c
     cudaError_t e = cudaFuncSetAttribute(k_conv_rowrun, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 5): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    k_conv_rowrun<<<static_cast<unsigned>(grid), THREADS, smem, st>>>(p, cfg, tm_y);
-    count_launch(1);
-    e = cudaGetLastError();
+    e = nmhost::launch_pdl(k_conv_rowrun, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_y);
+    nmhost::count_launch(1);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 5): %s", cudaGetErrorString(e));
     return NM_OK;
 }

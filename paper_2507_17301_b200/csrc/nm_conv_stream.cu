@@ -156,6 +156,8 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
+    pdl_launch_dependents();   // the next kernel may start its own set-up as SMs become free
+    pdl_wait();                // from here on global memory written by the previous kernel is read
 
     if (warp == 0) {
         // =========================== producer ===========================
@@ -492,9 +494,9 @@ nm_status_t launch(const ConvParams& p, const StreamCfg& cfg, cudaStream_t st)
                                          static_cast<int>(smem));
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 3): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    k_conv_stream<NK, MG><<<static_cast<unsigned>(grid), THREADS, smem, st>>>(p, cfg, tm_x, tm_w, tm_y);
+    e = nmhost::launch_pdl(k_conv_stream<NK, MG>, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x, tm_w, tm_y);
     nmhost::count_launch(1);
-    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_conv2d launch (variant 3): %s", cudaGetErrorString(e));
     return NM_OK;
 }

@@ -55,6 +55,27 @@ struct ConvParams {
 };
 
 namespace nmhost {
+// Launches `kernel` so that it may begin while the previous kernel of the stream drains
+// (programmatic dependent launch); the kernel orders itself with griddepcontrol.wait.
+// NM_NO_PDL=1 in the environment falls back to a plain launch.
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                       Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Sets the calling thread's error text and returns `s`.
 nm_status_t fail(nm_status_t s, const char* fmt, ...);
 void count_launch(int n = 1);

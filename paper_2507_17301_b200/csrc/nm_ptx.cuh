@@ -13,6 +13,14 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// ---- programmatic dependent launch -------------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start while the previous
+// kernel of the stream is still draining: everything before pdl_wait() (barrier set-up, TMEM
+// allocation, descriptor prefetch) then overlaps that tail.  pdl_wait() returns once the
+// previous kernel has completed and its writes are visible; without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier ---------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
