@@ -37,6 +37,10 @@ METRIC = "resnet50_conv_stack_images_per_s"
 UNIT = "images/s"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
+TF32_OVER_BF16 = 1.1 / 2.25   # nominal dense tensor peaks: 1.1 PFLOP/s TF32, 2.25 PFLOP/s bf16
+KERNEL_OF_VARIANT = {1: "k_conv_gather", 2: "k_conv_slab", 3: "k_conv_stream", 4: "k_conv_expand", 5: "k_conv_rowrun"}
+KERNEL_SOURCE = {"k_conv_gather": "nm_conv_gather.cu", "k_conv_slab": "nm_conv_slab.cu", "k_conv_stream": "nm_conv_stream.cu",
+                 "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu"}
 
 
 def peaks():
@@ -46,6 +50,36 @@ def peaks():
             d = json.load(f)
         return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]), "source": "measured"}
     return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "source": "fallback"}
+
+
+def source_digest(kernel: str) -> str:
+    """Digest of the kernel's source file: DRAM counters taken from an ncu capture are only quoted
+    while the kernel is unchanged since."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2507_17301_b200", "csrc", KERNEL_SOURCE[kernel])
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def recorded_traffic(kernel: str, batch: int):
+    """DRAM bytes (read + write) of one step's launches of `kernel`, from the committed summary of an
+    ncu capture (profiles/dram_traffic_<kernel>.txt: key = value lines), scaled to `batch`; None if
+    there is no summary or the kernel source has changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", f"dram_traffic_{kernel}.txt")
+    if not os.path.exists(path):
+        return None
+    kv = {}
+    with open(path) as f:
+        for line in f:
+            if "=" in line and not line.lstrip().startswith("#"):
+                k, v = line.split("=", 1)
+                kv[k.strip()] = v.strip()
+    try:
+        if kv["source_sha256_16"] != source_digest(kernel):
+            return None
+        return float(kv["dram_bytes_per_step"]) * batch / float(kv["batch"]), kv
+    except (KeyError, ValueError):
+        return None
 
 
 def algorithmic_bytes(s: inputs.ConvShape) -> int:
@@ -247,6 +281,8 @@ def main():
     ap.add_argument("--variant", type=int, default=None, help="force a kernel variant instead of auto-tuning")
     ap.add_argument("--bn", type=int, default=0, help="with --variant: output channels per CTA")
     ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
+    ap.add_argument("--save-plans", default=None, help="write the auto-tuned plans to this JSON file")
+    ap.add_argument("--load-plans", default=None, help="use the plans of this JSON file instead of auto-tuning")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -266,6 +302,10 @@ def main():
         layers = [s for s in layers if args.layer in s.name]
         assert layers, f"no layer matches {args.layer!r}"
     dev = torch.device("cuda", local if world > 1 else 0)
+    loaded = None
+    if args.load_plans:
+        with open(args.load_plans) as f:
+            loaded = json.load(f)
     state = []
     for li, s in enumerate(layers):
         w = inputs.make_weights(s, li).to(dev)
@@ -278,12 +318,19 @@ def main():
             x[b0:b0 + 8] = torch.randn((min(8, s.batch - b0), s.h, s.w, s.c_in), generator=g).to(dev)
         bias = inputs.make_bias(s, li).to(dev)
         y = torch.empty((s.batch, s.ho, s.wo, s.c_out), dtype=torch.float32, device=dev)
-        if args.variant is None:
+        if loaded is not None and s.name in loaded:
+            plan = nm.nm_plan_t()
+            plan.variant, plan.bn, plan.stages, plan.split = (loaded[s.name][k] for k in ("variant", "bn", "stages", "split"))
+        elif args.variant is None:
             plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
         else:
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.stages = args.variant, args.bn, args.stages
         state.append((s, hnd, x, bias, y, plan))
+
+    if args.save_plans and rank == 0:
+        with open(args.save_plans, "w") as f:
+            json.dump({s.name: plan.as_dict() for s, _, _, _, _, plan in state}, f, indent=1)
 
     def step():
         for s, hnd, x, bias, y, plan in state:
@@ -295,8 +342,11 @@ def main():
     sampler = ClockSampler(local if world > 1 else 0)
     if rank == 0:
         sampler.start()
-    launches0 = nm.nm_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if not args.no_extras:
+        for _ in range(200):   # about half a second of untimed steps so that the clock sampler sees the load
+            step()
+    launches0 = nm.nm_launch_count()
     barrier(world)
     e0.record()
     for _ in range(args.steps):
@@ -320,7 +370,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": "resnet50_conv_stack_b64_224_2of4" + (f" [only {args.layer}]" if args.layer else ""),
                    "layers": len(layers), "batch_per_gpu": args.batch,
-                   "tile_t": 64, "cache": "inputs larger than L2 (5.4 GB touched per step, one buffer per layer)",
+                   "tile_t": 64, "plans": "per layer by nm_autotune" if args.variant is None and not args.load_plans else "given", "cache": "inputs larger than L2 (5.4 GB touched per step, one buffer per layer)",
                    "parallelism": f"replicas x{world}"},
         "useful_tflops": flops_step / (ms_step * 1e-3) / 1e12,
         "gpu_launches": int(launches),
@@ -331,8 +381,12 @@ def main():
     }
 
     if rank == 0 and not args.no_extras and world == 1:
-        tf32_peak = measure_tf32_peak()
-        out["tf32_peak_tflops_measured"] = tf32_peak
+        # tensor roof: the measured bf16 GEMM peak scaled by the nominal TF32 : bf16 ratio; the library
+        # TF32 GEMM timed here is context
+        tf32_peak = pk["bf16_tflops"] * TF32_OVER_BF16
+        out["tf32_peak_tflops"] = tf32_peak
+        out["tf32_peak_source"] = f"{pk['source']} bf16 GEMM peak x nominal TF32/bf16 ratio (1.1 / 2.25)"
+        out["tf32_cublas_tflops_measured"] = measure_tf32_peak()
         # per-layer pass: events around each launch, other layers' traffic in between keeps it cold
         reps = 5
         per = [[] for _ in state]
@@ -360,7 +414,35 @@ def main():
                           "bound": "tensor" if t_tc > t_hbm else "hbm", "roofline_frac": round(t_roof / ms, 3),
                           "plan": plan.as_dict()})
         out["stack_roofline_frac"] = t_roof_sum / ms_step
+        out["stack_roofline_note"] = ("sum over layers of max(kept FLOPs / TF32 peak, algorithmic bytes / HBM peak) "
+                                      "divided by the measured time of a step")
         out["per_layer"] = table
+        # roofline object: the kernel that takes the largest share of a step, over all its launches
+        by_kernel = {}
+        for (s, hnd, x, bias, y, plan), row in zip(state, table):
+            k = KERNEL_OF_VARIANT.get(plan.variant, "library default")
+            acc = by_kernel.setdefault(k, {"ms": 0.0, "bytes": 0, "flops": 0, "launches": 0})
+            acc["ms"] += row["ms"]
+            acc["bytes"] += algorithmic_bytes(s)
+            acc["flops"] += useful_flops(s)
+            acc["launches"] += 1
+        total_ms = sum(v["ms"] for v in by_kernel.values())
+        out["kernel_shares"] = {k: {"launches": v["launches"], "ms": round(v["ms"], 4), "share": round(v["ms"] / total_ms, 3)}
+                                for k, v in by_kernel.items()}
+        dom = max(by_kernel, key=lambda k: by_kernel[k]["ms"])
+        d = by_kernel[dom]
+        dom_gbs = d["bytes"] / (d["ms"] * 1e-3) / 1e9
+        traffic = recorded_traffic(dom, args.batch) if dom in KERNEL_SOURCE and not args.layer else None
+        out["roofline"] = {
+            "bound": "hbm", "achieved": dom_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": dom_gbs / pk["hbm_gbs"],
+            "traffic": traffic[0] / d["launches"] if traffic else None,
+            "peak_source": pk["source"] + " (burst copy figure; each launch is timed alone between events)",
+            "kernel": dom, "launches_per_step": d["launches"], "avg_launch_ms": d["ms"] / d["launches"],
+            "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],
+            "share_of_step": d["ms"] / total_ms,
+            "useful_tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12,
+            "note": "algorithmic bytes of the layers this kernel runs / their summed launch times (median of 5 per layer)",
+        }
 
         # cuDNN dense convolution on the same shapes (context, unpruned weights, TF32 allowed)
         try:
