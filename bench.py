@@ -175,11 +175,21 @@ def barrier(world):
     torch.cuda.synchronize()
 
 
-def max_over_ranks(value: float, world: int) -> float:
+def replica_seed(layer: int, rank: int) -> int:
+    """Seed of a replica's activations for one layer: every rank draws its own batch."""
+    return 1 + 1000 * layer + 7919 * rank
+
+
+def aggregate_images_per_s(batch_per_gpu: int, world: int, ms_step_max: float) -> float:
+    """Whole-job throughput of `world` replicas: all images of a step over the slowest rank's step time."""
+    return world * batch_per_gpu / (ms_step_max * 1e-3)
+
+
+def max_over_ranks(value: float, world: int, device: str = "cuda") -> float:
     if world == 1:
         return value
     import torch.distributed as dist
-    t = torch.tensor([value], dtype=torch.float64, device="cuda")
+    t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
 
@@ -311,7 +321,7 @@ def main():
         w = inputs.make_weights(s, li).to(dev)
         hnd = nm.nm_prune(w, s.n_keep, s.m_group, s.tile_t)
         del w
-        g = torch.Generator(device="cpu").manual_seed(1 + 1000 * li + 7919 * rank)
+        g = torch.Generator(device="cpu").manual_seed(replica_seed(li, rank))
         # activations ~ N(0,1): drawn on the host in slices to bound pinned/pageable staging
         x = torch.empty((s.batch, s.h, s.w, s.c_in), dtype=torch.float32, device=dev)
         for b0 in range(0, s.batch, 8):
@@ -359,7 +369,7 @@ def main():
     for s, hnd, *_ in state:
         nm.nm_weights_check(hnd)
     ms_step = ms_total / args.steps
-    value = world * args.batch / (ms_step * 1e-3)
+    value = aggregate_images_per_s(args.batch, world, ms_step)
 
     bytes_step = sum(algorithmic_bytes(s) for s in layers)
     flops_step = sum(useful_flops(s) for s in layers)

@@ -55,12 +55,26 @@ typedef struct nm_weights nm_weights_t;
 
 /*
  * Launch plan for nm_conv2d (the analogue of the paper's per-layer template parameters, Sec. 3.3).
- *   variant  0 = let the library choose; 1 = direct-gather kernel (any shape);
- *            2 = slab kernel (dense activation slab staged once per CTA, compacted on chip;
- *                needs c_in % 4 == 0 and m_group | 32-column slab, see nm_conv2d)
- *   bn       output channels per CTA (a multiple of the weights' tile_t), 0 = default
+ *   variant  0 = let the library choose;
+ *            1 = direct-gather kernel (any shape);
+ *            2 = slab kernel (dense activation slab staged once per CTA, kept columns picked by
+ *                4-byte loads; needs c_in % 4 == 0 and whole N:M groups per slab);
+ *            3 = stream kernel (persistent; slab read once with 16-byte loads, kept columns of
+ *                every tile selected in registers; needs c_in % 32 == 0, tile_t % 16 == 0,
+ *                c_out % tile_t == 0, N:M one of 1:4 2:4 3:4 1:8 2:8 4:8 or N = M, an input of at
+ *                least 128 KiB);
+ *            4 = expanded-operand kernel (persistent; the slab feeds the tensor core directly and
+ *                zero weights stand for the pruned columns: M/N times the kept FLOPs, no
+ *                per-element work; needs c_in % 32 == 0, c_out % 32 == 0, an input of at least
+ *                128 KiB; any tile_t, any N:M);
+ *            5 = row-run kernel for few input channels (c_in % 32 != 0, dil_w = 1, output rows of
+ *                at most 128 pixels, K <= 512, c_out % 32 == 0 and <= 256, w * c_in * 4 a multiple
+ *                of 16).
+ *   bn       output channels per CTA / work item (variants 2, 3: a multiple of tile_t; variant 4: a
+ *            multiple of 32 up to 256), 0 = default
  *   stages   depth of the shared-memory ring, 0 = default
- *   split    reserved, 0
+ *   split    variant 2 only: 1 = cp.async producer, 2 = direct-store epilogue; otherwise 0
+ * A plan the layer does not admit gives NM_ERR_UNSUPPORTED.
  */
 typedef struct {
     int variant;
@@ -163,8 +177,8 @@ nm_status_t nm_weights_free(nm_weights_t* w);
  *                          x[n][oh*stride_h - pad_h + kh_j*dil_h][ow*stride_w - pad_w + kw_j*dil_w][c_j] )
  * with (kh_j, kw_j, c_j) decoded from indices[o / tile_t][j] and reads outside the image = 0.
  * Arithmetic: operands rounded to TF32 (weights once at prune time, round-to-nearest; activations
- * round-to-nearest where they pass through registers, truncated where the staged slab feeds the
- * tensor core directly), products accumulated in fp32.
+ * round-to-nearest where they pass through registers (variants 1-3), truncated where the staged
+ * slab feeds the tensor core directly (variants 4, 5)), products accumulated in fp32.
  *
  *   x      device fp32 [batch][h][wd][c_in]      bias  device fp32 [c_out] or NULL
  *   y      device fp32 [batch][ho][wo][c_out]    relu  0 = identity, 1 = ReLU
