@@ -4,14 +4,16 @@
 //
 // With NHWC activations and dil_w = 1, the (kw, c) part of a patch row is ONE contiguous run of
 // kw * c_in floats of the input row.  One work item is one output row (at most 128 pixels):
-//   producer (1 thread)    bulk-copies the kh input rows the item needs into shared memory (rows
-//                          outside the image are replaced by a row of zeros, left / right padding by
-//                          zeroed margins of the row buffers);
+//   producer (1 thread)    bulk-copies the kh input rows the item needs into shared memory: with
+//                          dil_h = 1 they are adjacent in memory, so ONE copy brings them all (rows
+//                          outside the image are simply not copied);
 //   builders (8 warps)     lay the patch matrix [128 pixels x K] down in 32-column sub-tiles in the
 //                          K-major, 128-byte-swizzled layout the tensor core reads: lane = column,
 //                          so a warp reads 32 consecutive floats of a run and writes one 128-byte
-//                          row, both free of bank conflicts (tile rows past the end of the output
-//                          row are filled with zeros).  This is the fused im2col + packing of
+//                          row, both free of bank conflicts.  Padding is resolved per column with a
+//                          precomputed range of valid output pixels (outside it, past the end of
+//                          the output row and for kernel rows outside the image the builders write
+//                          zeros).  This is the fused im2col + packing of
 //                          Sec. 3.2 done in shared memory; nothing of it reaches global memory;
 //   MMA issuer (1 thread)  four 128 x C_out x 8 TF32 tcgen05.mma per sub-tile against the weights,
 //                          which stay resident in shared memory for the whole kernel (expanded
@@ -38,8 +40,7 @@ constexpr int MAX_KB = 16;   // sub-tiles of 32 columns: K <= 512
 struct RowCfg {
     int nkb;          // ceil(K / 32)
     int run;          // kw * c_in: contiguous floats per kernel row
-    int pitch;        // floats per row buffer (margins included)
-    int leftpad;      // floats of zero margin before the row body (multiple of 4)
+    int pitch;        // floats per row buffer = w * c_in
     int row_bytes;    // w * c_in * 4
     int bn;           // = c_out
     int w_bytes;      // nkb * bn * 128
@@ -57,13 +58,14 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
     __shared__ int s_koff[MAX_KB * 32];   // per column: kernel row << 24 | float offset inside the row set; -1 = padding
+    __shared__ uint32_t s_range[MAX_KB * 32];   // per column: first valid output pixel << 16 | number of valid ones
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t w_smem = base;
     const uint32_t a_ring = w_smem + ((cfg.w_bytes + 1023) / 1024) * 1024;
     const uint32_t staging = a_ring + A_RING * SUB_BYTES;
-    const uint32_t rowbuf = staging + STAGING_BYTES;                 // two row sets, then one row of zeros
+    const uint32_t rowbuf = staging + STAGING_BYTES;                 // two row sets, then 16 bytes of zeros
     const uint32_t zero_row = rowbuf + 2 * cfg.rowset_bytes;
     volatile int* abort_flag = &s_abort;
 
@@ -84,17 +86,24 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         s_abort = 0;
         tma_prefetch_desc(&tm_y);
     }
-    // margins of the row buffers and the zero row: cleared once, never written again
+    // per-column tables, and the word of zeros every invalid element is read from
     {
-        const int words = (2 * cfg.rowset_bytes + cfg.pitch * 4) / 4;
-        for (int i = tid; i < words; i += THREADS)
-            asm volatile("st.shared.u32 [%0], %1;" ::"r"(rowbuf + i * 4), "r"(0u) : "memory");
+        if (tid < 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(zero_row + tid * 4), "r"(0u) : "memory");
         for (int i = tid; i < cfg.nkb * 32; i += THREADS) {
             const int khi = i / cfg.run;
-            s_koff[i] = i < p.k ? ((khi << 24) | (khi * cfg.pitch + (i - khi * cfg.run))) : -1;
+            const int kr = i - khi * cfg.run;          // position inside the run: kw * c_in + c
+            const int kwi = (kr / p.c_in) * p.dil_w;   // (dil_w = 1)
+            s_koff[i] = i < p.k ? ((khi << 24) | (khi * cfg.pitch + kr)) : -1;
+            // output pixels ow with 0 <= ow * stride_w - pad_w + kwi < w, clipped to the output row
+            int lo = p.pad_w - kwi;
+            lo = lo > 0 ? (lo + p.stride_w - 1) / p.stride_w : 0;
+            int hi = p.w + p.pad_w - 1 - kwi;
+            hi = hi >= 0 ? hi / p.stride_w : -1;
+            if (hi > p.wo - 1) hi = p.wo - 1;
+            const int cnt = hi >= lo ? hi - lo + 1 : 0;
+            s_range[i] = (static_cast<uint32_t>(lo) << 16) | static_cast<uint32_t>(cnt);
         }
     }
-    fence_proxy_async();   // the zeroed buffers are later written by bulk copies (async proxy)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -114,19 +123,31 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                 const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
                 if (wrapped && !mbar_wait(smem_u32(&s_rfree[set]), par ^ 1u)) { *abort_flag = 2; break; }
                 const int ih0 = oh * p.stride_h - p.pad_h;
-                int valid = 0;
-                for (int r = 0; r < p.kh; ++r) {
-                    const int ih = ih0 + r * p.dil_h;
-                    valid += (ih >= 0 && ih < p.h) ? 1 : 0;
-                }
                 const uint32_t bar = smem_u32(&s_rfull[set]);
-                mbar_arrive_expect_tx(bar, static_cast<uint32_t>(valid) * cfg.row_bytes);
-                for (int r = 0; r < p.kh; ++r) {
-                    const int ih = ih0 + r * p.dil_h;
-                    if (ih >= 0 && ih < p.h)
-                        bulk_load_1d(rowbuf + set * cfg.rowset_bytes + (r * cfg.pitch + cfg.leftpad) * 4,
-                                     p.x + (static_cast<size_t>(n) * p.h + ih) * p.w * p.c_in,
-                                     static_cast<uint32_t>(cfg.row_bytes), bar);
+                const uint32_t dst0 = rowbuf + set * cfg.rowset_bytes;
+                const float* img = p.x + static_cast<size_t>(n) * p.h * p.w * p.c_in;
+                if (p.dil_h == 1) {
+                    // the kernel rows are adjacent input rows: one copy of the ones inside the image
+                    const int first = ih0 > 0 ? ih0 : 0;
+                    const int last = ih0 + p.kh - 1 < p.h - 1 ? ih0 + p.kh - 1 : p.h - 1;
+                    const int cnt = last >= first ? last - first + 1 : 0;
+                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(cnt) * cfg.row_bytes);
+                    if (cnt > 0)
+                        bulk_load_1d(dst0 + (first - ih0) * cfg.row_bytes, img + static_cast<size_t>(first) * p.w * p.c_in,
+                                     static_cast<uint32_t>(cnt) * cfg.row_bytes, bar);
+                } else {
+                    int valid = 0;
+                    for (int r = 0; r < p.kh; ++r) {
+                        const int ih = ih0 + r * p.dil_h;
+                        valid += (ih >= 0 && ih < p.h) ? 1 : 0;
+                    }
+                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(valid) * cfg.row_bytes);
+                    for (int r = 0; r < p.kh; ++r) {
+                        const int ih = ih0 + r * p.dil_h;
+                        if (ih >= 0 && ih < p.h)
+                            bulk_load_1d(dst0 + r * cfg.row_bytes, img + static_cast<size_t>(ih) * p.w * p.c_in,
+                                         static_cast<uint32_t>(cfg.row_bytes), bar);
+                    }
                 }
                 ++issued;
                 if (set == 1) { par ^= 1u; wrapped = true; }
@@ -241,26 +262,27 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
                 if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
                 const int ko = s_koff[j * 32 + lane];
-                uint32_t src = zero_row;           // padding column or a kernel row outside the image
-                int step = 0;                      // bytes between two pixels of this column
+                const uint32_t rng = s_range[j * 32 + lane];
+                const int lo = static_cast<int>(rng >> 16);
+                uint32_t cnt = 0;                  // valid output pixels of this column: lo .. lo + cnt - 1
+                uint32_t src = zero_row;
                 if (ko >= 0) {
                     const int khi = ko >> 24;
                     const int ih = ih0 + khi * p.dil_h;
-                    if (ih >= 0 && ih < p.h) {
-                        src = rows + ((ko & 0xFFFFFF) + cfg.leftpad - p.pad_w * p.c_in) * 4;
-                        step = p.stride_w * p.c_in * 4;
-                    }
+                    if (ih >= 0 && ih < p.h) cnt = rng & 0xFFFFu;
+                    // element of output pixel 0 (before the row's start for padded columns: never read there)
+                    src = rows + ((ko & 0xFFFFFF) - p.pad_w * p.c_in) * 4;
                 }
+                const int step8 = p.stride_w * p.c_in * 4 * 8;   // bytes between pixels ow and ow + 8
                 // rows bw, bw + 8, ...: (row % 8) is the same for all of them, so is the swizzle term
                 uint32_t dst = a_ring + rp.s * SUB_BYTES + ((lane & 3) << 2) + bw * 128 +
                                ((static_cast<uint32_t>(lane >> 2) ^ static_cast<uint32_t>(bw)) << 4);
-                src += bw * step;
-                const int step8 = step * 8;
+                src += bw * (step8 >> 3);
                 uint32_t v[BM / 8];
 #pragma unroll
                 for (int i = 0; i < BM / 8; ++i) {
-                    // tile rows past the end of the output row read the row of zeros
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(bw + i * 8 < p.wo ? src : zero_row));
+                    const bool valid = static_cast<uint32_t>(bw + i * 8 - lo) < cnt;
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(valid ? src : zero_row));
                     src += step8;
                 }
 #pragma unroll
@@ -315,14 +337,9 @@ bool make_cfg(const ConvParams& p, RowCfg* cfg, size_t* smem_out)
     cfg->nkb = (p.k + 31) / 32;
     if (cfg->nkb > MAX_KB) return false;
     cfg->run = p.kw * p.c_in;
-    cfg->leftpad = ((p.pad_w * p.c_in + 3) / 4) * 4;
-    // furthest float a pixel of the output row can touch, counted from the start of the row body
-    // (tile rows past the end of the output row read the row of zeros instead)
-    const long long reach = (static_cast<long long>(p.wo - 1) * p.stride_w - p.pad_w + p.kw) * p.c_in;
-    const long long body = static_cast<long long>(p.w) * p.c_in;
-    const long long pitch = cfg->leftpad + (reach > body ? reach : body);
-    cfg->pitch = static_cast<int>(((pitch + 3) / 4) * 4);
-    if (cfg->pitch > 16384) return false;
+    cfg->pitch = p.w * p.c_in;
+    if (static_cast<long long>(p.kh) * p.w * p.c_in * 4 >= (1 << 20)) return false;   // one copy, one mbarrier phase
+    if (p.wo > 0xFFFF) return false;
     cfg->row_bytes = p.w * p.c_in * 4;
     cfg->bn = p.c_out;
     cfg->w_bytes = cfg->nkb * cfg->bn * 128;
@@ -330,7 +347,7 @@ bool make_cfg(const ConvParams& p, RowCfg* cfg, size_t* smem_out)
     cfg->n_work = static_cast<long long>(p.batch) * p.ho;
     if (static_cast<long long>(p.batch) * p.ho >= (1ll << 31)) return false;
     const size_t smem = 1024 + static_cast<size_t>((cfg->w_bytes + 1023) / 1024) * 1024 + A_RING * SUB_BYTES + STAGING_BYTES +
-                        2 * static_cast<size_t>(cfg->rowset_bytes) + static_cast<size_t>(cfg->pitch) * 4;
+                        2 * static_cast<size_t>(cfg->rowset_bytes) + 16;
     if (smem > 227 * 1024 - 4096) return false;
     *smem_out = smem < 120 * 1024 ? 120 * 1024 : smem;
     return true;
