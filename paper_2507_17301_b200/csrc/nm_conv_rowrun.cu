@@ -32,7 +32,8 @@ using namespace nmk;
 
 constexpr int BM = 128;
 constexpr int SUB_BYTES = BM * 128;
-constexpr int A_RING = 6;
+constexpr int A_RING = 4;
+constexpr int MAX_SETS = 4;   // row sets in flight: the copy of item i + n_sets - 1 is issued while item i is built
 constexpr int THREADS = 512;
 constexpr int STAGING_BYTES = 4 * 2 * 4096;
 constexpr int MAX_KB = 16;   // sub-tiles of 32 columns: K <= 512
@@ -45,6 +46,7 @@ struct RowCfg {
     int bn;           // = c_out
     int w_bytes;      // nkb * bn * 128
     int rowset_bytes; // kh * pitch * 4
+    int n_sets;       // row sets in the ring (2 .. MAX_SETS)
     long long n_work; // batch * ho
 };
 
@@ -54,7 +56,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUtensorMap tm_y)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t s_wfull, s_rfull[2], s_rfree[2], s_afull[A_RING], s_afree[A_RING], s_accfull[2], s_accfree[2];
+    __shared__ uint64_t s_wfull, s_rfull[MAX_SETS], s_rfree[MAX_SETS], s_afull[A_RING], s_afree[A_RING], s_accfull[2], s_accfree[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
     __shared__ int s_koff[MAX_KB * 32];   // per column: kernel row << 24 | float offset inside the row set; -1 = padding
@@ -66,15 +68,17 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
     const uint32_t a_ring = w_smem + ((cfg.w_bytes + 1023) / 1024) * 1024;
     const uint32_t staging = a_ring + A_RING * SUB_BYTES;
     const uint32_t rowbuf = staging + STAGING_BYTES;                 // two row sets, then 16 bytes of zeros
-    const uint32_t zero_row = rowbuf + 2 * cfg.rowset_bytes;
+    const uint32_t zero_row = rowbuf + cfg.n_sets * cfg.rowset_bytes;
     volatile int* abort_flag = &s_abort;
 
     if (warp == 2) tmem_alloc(smem_u32(&s_tmem), 512);
     if (tid == 0) {
         mbar_init(smem_u32(&s_wfull), 1);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < MAX_SETS; ++i) {
             mbar_init(smem_u32(&s_rfull[i]), 1);
             mbar_init(smem_u32(&s_rfree[i]), 8);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&s_accfull[i]), 1);
             mbar_init(smem_u32(&s_accfree[i]), 4);
         }
@@ -116,15 +120,14 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         if (lane == 0) {
             mbar_arrive_expect_tx(smem_u32(&s_wfull), static_cast<uint32_t>(cfg.w_bytes));
             bulk_load_1d(w_smem, p.wx, static_cast<uint32_t>(cfg.w_bytes), smem_u32(&s_wfull));
-            uint32_t set = 0, par = 0;
-            bool wrapped = false;
+            RingPos rs;
             int issued = 0;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
                 const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
-                if (wrapped && !mbar_wait(smem_u32(&s_rfree[set]), par ^ 1u)) { *abort_flag = 2; break; }
+                if (rs.wrapped && !mbar_wait(smem_u32(&s_rfree[rs.s]), rs.parity ^ 1u)) { *abort_flag = 2; break; }
                 const int ih0 = oh * p.stride_h - p.pad_h;
-                const uint32_t bar = smem_u32(&s_rfull[set]);
-                const uint32_t dst0 = rowbuf + set * cfg.rowset_bytes;
+                const uint32_t bar = smem_u32(&s_rfull[rs.s]);
+                const uint32_t dst0 = rowbuf + rs.s * cfg.rowset_bytes;
                 const float* img = p.x + static_cast<size_t>(n) * p.h * p.w * p.c_in;
                 if (p.dil_h == 1) {
                     // the kernel rows are adjacent input rows: one copy of the ones inside the image
@@ -150,15 +153,14 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                     }
                 }
                 ++issued;
-                if (set == 1) { par ^= 1u; wrapped = true; }
-                set ^= 1u;
+                rs.advance(cfg.n_sets);
             }
             if (aborted(abort_flag)) {
                 (void)mbar_wait(smem_u32(&s_wfull), 0);
-                for (int back = 0; back < 2 && back < issued; ++back) {
-                    if (set == 0) par ^= 1u;
-                    set ^= 1u;
-                    (void)mbar_wait(smem_u32(&s_rfull[set]), par);
+                for (int back = 0; back < cfg.n_sets && back < issued; ++back) {
+                    if (rs.s == 0) { rs.s = cfg.n_sets; rs.parity ^= 1u; }
+                    --rs.s;
+                    (void)mbar_wait(smem_u32(&s_rfull[rs.s]), rs.parity);
                 }
             }
         }
@@ -249,14 +251,14 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         // =========================== builders ===========================
         const int bw = warp - 8;   // rows bw, bw + 8, ...
         RingPos rp;
-        uint32_t set = 0, set_par = 0;
+        RingPos rs;
         for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
             const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
             const int ih0 = oh * p.stride_h - p.pad_h;
-            bool ok = mbar_wait(smem_u32(&s_rfull[set]), set_par);
+            bool ok = mbar_wait(smem_u32(&s_rfull[rs.s]), rs.parity);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 3;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
-            const uint32_t rows = rowbuf + set * cfg.rowset_bytes;
+            const uint32_t rows = rowbuf + rs.s * cfg.rowset_bytes;
             for (int j = 0; j < cfg.nkb; ++j) {
                 ok = !rp.wrapped || mbar_wait(smem_u32(&s_afree[rp.s]), rp.parity ^ 1u);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
@@ -297,9 +299,8 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
             }
             if (aborted(abort_flag)) break;
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&s_rfree[set]));
-            if (set == 1) set_par ^= 1u;
-            set ^= 1u;
+            if (lane == 0) mbar_arrive(smem_u32(&s_rfree[rs.s]));
+            rs.advance(cfg.n_sets);
         }
     }
 
@@ -346,8 +347,10 @@ bool make_cfg(const ConvParams& p, RowCfg* cfg, size_t* smem_out)
     cfg->rowset_bytes = p.kh * cfg->pitch * 4;
     cfg->n_work = static_cast<long long>(p.batch) * p.ho;
     if (static_cast<long long>(p.batch) * p.ho >= (1ll << 31)) return false;
-    const size_t smem = 1024 + static_cast<size_t>((cfg->w_bytes + 1023) / 1024) * 1024 + A_RING * SUB_BYTES + STAGING_BYTES +
-                        2 * static_cast<size_t>(cfg->rowset_bytes) + 16;
+    const size_t fixed = 1024 + static_cast<size_t>((cfg->w_bytes + 1023) / 1024) * 1024 + A_RING * SUB_BYTES + STAGING_BYTES + 16;
+    cfg->n_sets = MAX_SETS;
+    while (cfg->n_sets > 2 && fixed + static_cast<size_t>(cfg->n_sets) * cfg->rowset_bytes > 227 * 1024 - 4096) --cfg->n_sets;
+    const size_t smem = fixed + static_cast<size_t>(cfg->n_sets) * cfg->rowset_bytes;
     if (smem > 227 * 1024 - 4096) return false;
     *smem_out = smem < 120 * 1024 ? 120 * 1024 : smem;
     return true;
