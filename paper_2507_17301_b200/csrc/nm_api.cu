@@ -142,6 +142,8 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
             return nmhost::launch_conv_expand(p, plan, st);
         case 5:
             return nmhost::launch_conv_rowrun(p, plan, st);
+        case 6:
+            return nmhost::launch_conv_window(p, plan, st);
         default:
             return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
     }
@@ -152,6 +154,13 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
 {
     std::vector<nm_plan_t> out;
     nm_plan_t a;
+    std::memset(&a, 0, sizeof(a));
+    for (int mt : {1, 2}) {                 // window kernel (stride-1 spatial kernels)
+        for (int bn : {64, 128, 256}) {
+            a.variant = 6; a.bn = bn; a.split = mt; a.stages = 0;
+            if (nmhost::window_plan_ok(p, &a)) out.push_back(a);
+        }
+    }
     std::memset(&a, 0, sizeof(a));
     a.variant = 5;                          // row-run kernel (few input channels)
     if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, &a)) out.push_back(a);

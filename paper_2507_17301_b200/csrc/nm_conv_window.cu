@@ -1,0 +1,439 @@
+// Variant 6: window kernel — stride-1 convolutions with a spatial kernel (3x3 and the like) as an
+// implicit GEMM whose taps are SHIFTED VIEWS of one input patch held in shared memory.
+//
+// The im2col form re-reads every input element once per tap (nine 128-byte rows per pixel and
+// 32-channel block through the TMA unit).  Here one tiled TMA load brings, per 32-channel block,
+// the patch [R + (kh-1)*dil rows x Wp = W + 2*pad columns] once, zero-filled outside the image,
+// in the 128-byte-swizzled layout: one 128-byte row per patch pixel.  Output positions are
+// numbered along the PADDED width (position = row * Wp + column), so the A operand of tap (i, j)
+// for 128 consecutive positions is simply the 128 patch rows that start (i*dil_h*Wp + j*dil_w)
+// rows further down: the same shared-memory bytes, another descriptor start address.  Positions
+// whose column falls in the padding produce junk rows that are never stored.
+//
+//   patch producer (1 thread)   one 4-D tiled TMA load per 32-channel block and work item
+//   weight producer (1 thread)  one contiguous bulk copy per (32-channel block, tap): the
+//                               expanded, pre-swizzled weights [BN x 32] (zeros = pruned columns)
+//   MMA issuer (1 thread)       per block and tap four 128 x BN x 8 TF32 tcgen05.mma per M-tile
+//   epilogue (4 warps)          TMEM -> registers, + bias, ReLU, staging in output-row order, one TMA
+//                               store per output row and 32-channel block
+// A work item is (image, block of R output rows, BN channels) with R * Wp <= 128 * MT positions
+// (MT = 1 or 2 M-tiles sharing patch and weights).  Persistent CTAs, static schedule, bounded waits.
+#include "nm_internal.h"
+#include "nm_ptx.cuh"
+#include "nm_tmap.cuh"
+
+namespace {
+
+using namespace nmk;
+
+constexpr int BM = 128;
+constexpr int THREADS = 256;
+constexpr int MAX_P = 4;    // patch ring slots
+constexpr int MAX_W = 12;   // weight ring slots
+
+struct WinCfg {
+    int bn, n_slices;
+    int mt;            // M-tiles per item (1 or 2)
+    int r_rows;        // output rows per item
+    int wp;            // padded width = positions per output row
+    int wp8;           // staging rows per output row (wp rounded up to 8)
+    int pr;            // patch rows = r_rows + (kh - 1) * dil_h
+    int patch_bytes;   // TMA box bytes = pr * wp * 128
+    int pslot_bytes;   // patch slot incl. overrun rows, multiple of 1024
+    int n_p, n_w;      // ring depths
+    int n_kb;          // c_in / 32
+    int row_blocks;    // ceil(ho / r_rows)
+    int stage_bytes;   // one staging buffer = r_rows * wp8 * 128
+    long long n_work;
+};
+
+__device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
+
+__device__ __forceinline__ void tma_load_tiled_4d(uint32_t dst, const void* tmap, uint32_t bar, int c, int w, int h, int n)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const void* tmap, uint32_t src, int c, int w, int h, int n)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tmap),
+                 "r"(src), "r"(c), "r"(w), "r"(h), "r"(n)
+                 : "memory");
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier of the 128 epilogue threads that also ORs a flag, so that all of them take the same exit.
+__device__ __forceinline__ bool epi_bar_or(bool flag)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pin, pout;\n\t"
+        "setp.ne.u32 pin, %1, 0;\n\t"
+        "bar.red.or.pred pout, 1, 128, pin;\n\t"
+        "selp.u32 %0, 1, 0, pout;\n\t"
+        "}\n"
+        : "=r"(out)
+        : "r"(flag ? 1u : 0u)
+        : "memory");
+    return out != 0;
+}
+
+// K-major, 128-byte-swizzled operand whose first row may sit on any 128-byte boundary of a
+// 1024-byte-aligned buffer: the tensor core derives the swizzle phase of a row from its
+// shared-memory address (as the TMA unit did when it wrote the row), so a view shifted by whole
+// rows needs nothing but another start address (checked bit for bit by the integer-valued tests).
+__device__ __forceinline__ uint64_t desc_rows(uint32_t addr) { return umma_desc_k_sw128(addr, 1024); }
+
+struct ItemPos {
+    int slice, n, oh0;
+};
+__device__ __forceinline__ ItemPos item_of(long long work, const WinCfg& cfg)
+{
+    ItemPos it;
+    it.slice = static_cast<int>(work % cfg.n_slices);
+    const long long rest = work / cfg.n_slices;
+    const int rb = static_cast<int>(rest % cfg.row_blocks);
+    it.n = static_cast<int>(rest / cfg.row_blocks);
+    it.oh0 = rb * cfg.r_rows;
+    return it;
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUtensorMap tm_x,
+              const __grid_constant__ CUtensorMap tm_y)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t s_pfull[MAX_P], s_pfree[MAX_P], s_wfull[MAX_W], s_wfree[MAX_W], s_accfull[2], s_accfree[2];
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t p_ring = base;
+    const uint32_t w_ring = p_ring + cfg.n_p * cfg.pslot_bytes;
+    const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
+    const uint32_t wslot_bytes = (w_bytes + 1023u) & ~1023u;
+    const uint32_t staging = w_ring + cfg.n_w * wslot_bytes;
+    const int n_taps = p.kh * p.kw;
+    const int acc_cols = cfg.mt * cfg.bn;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == 2) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (tid == 0) {
+        for (int i = 0; i < MAX_P; ++i) { mbar_init(smem_u32(&s_pfull[i]), 1); mbar_init(smem_u32(&s_pfree[i]), 1); }
+        for (int i = 0; i < MAX_W; ++i) { mbar_init(smem_u32(&s_wfull[i]), 1); mbar_init(smem_u32(&s_wfree[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&s_accfull[i]), 1); mbar_init(smem_u32(&s_accfree[i]), 4); }
+        mbar_fence_init();
+        s_abort = 0;
+        tma_prefetch_desc(&tm_x);
+        tma_prefetch_desc(&tm_y);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    pdl_launch_dependents();
+    pdl_wait();
+
+    if (warp == 0) {
+        // =========================== patch producer ===========================
+        if (lane == 0) {
+            RingPos rp;
+            int issued = 0;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+                const ItemPos it = item_of(work, cfg);
+                for (int kb = 0; kb < cfg.n_kb; ++kb) {
+                    if (rp.wrapped && !mbar_wait(smem_u32(&s_pfree[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
+                    if (aborted(abort_flag)) break;
+                    const uint32_t bar = smem_u32(&s_pfull[rp.s]);
+                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(cfg.patch_bytes));
+                    tma_load_tiled_4d(p_ring + rp.s * cfg.pslot_bytes, &tm_x, bar, kb * 32, -p.pad_w, it.oh0 - p.pad_h, it.n);
+                    rp.advance(cfg.n_p);
+                    ++issued;
+                }
+            }
+            if (aborted(abort_flag)) {
+                for (int back = 0; back < cfg.n_p && back < issued; ++back) {
+                    if (rp.s == 0) { rp.s = cfg.n_p; rp.parity ^= 1u; }
+                    --rp.s;
+                    (void)mbar_wait(smem_u32(&s_pfull[rp.s]), rp.parity);
+                }
+            }
+        }
+    } else if (warp == 3) {
+        // =========================== weight producer ===========================
+        if (lane == 0) {
+            RingPos rw;
+            int issued = 0;
+            const size_t blk_floats = static_cast<size_t>(p.c_out) * 32;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+                const ItemPos it = item_of(work, cfg);
+                const float* w0 = p.wx + static_cast<size_t>(it.slice) * cfg.bn * 32;
+                for (int kb = 0; kb < cfg.n_kb && !aborted(abort_flag); ++kb) {
+                    const float* wsrc = w0 + static_cast<size_t>(kb) * blk_floats;   // tap 0 of this channel block
+                    for (int t = 0; t < n_taps; ++t) {
+                        if (rw.wrapped && !mbar_wait(smem_u32(&s_wfree[rw.s]), rw.parity ^ 1u)) *abort_flag = 9;
+                        if (aborted(abort_flag)) break;
+                        const uint32_t bar = smem_u32(&s_wfull[rw.s]);
+                        mbar_arrive_expect_tx(bar, w_bytes);
+                        bulk_load_1d(w_ring + rw.s * wslot_bytes, wsrc, w_bytes, bar);
+                        wsrc += static_cast<size_t>(cfg.n_kb) * blk_floats;          // same channels, next tap
+                        rw.advance(cfg.n_w);
+                        ++issued;
+                    }
+                }
+            }
+            if (aborted(abort_flag)) {
+                for (int back = 0; back < cfg.n_w && back < issued; ++back) {
+                    if (rw.s == 0) { rw.s = cfg.n_w; rw.parity ^= 1u; }
+                    --rw.s;
+                    (void)mbar_wait(smem_u32(&s_wfull[rw.s]), rw.parity);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
+            RingPos rp, rw;
+            uint32_t ab = 0, acc_par = 0;
+            bool acc_wrapped = false;
+            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+                if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem + ab * acc_cols;
+                for (int kb = 0; kb < cfg.n_kb && !aborted(abort_flag); ++kb) {
+                    if (!mbar_wait(smem_u32(&s_pfull[rp.s]), rp.parity)) { *abort_flag = 6; break; }
+                    const uint32_t patch = p_ring + rp.s * cfg.pslot_bytes;
+                    int ti = 0, tj = 0;
+                    for (int t = 0; t < n_taps; ++t) {
+                        if (!mbar_wait(smem_u32(&s_wfull[rw.s]), rw.parity)) { *abort_flag = 7; break; }
+                        tc_fence_after();
+                        const uint32_t wsl = w_ring + rw.s * wslot_bytes;
+                        const uint32_t rowoff = static_cast<uint32_t>(ti * p.dil_h * cfg.wp + tj * p.dil_w) * 128u;
+                        for (int m = 0; m < cfg.mt; ++m) {
+                            const uint32_t a_addr = patch + static_cast<uint32_t>(m) * (BM * 128u) + rowoff;
+#pragma unroll
+                            for (int kq = 0; kq < 4; ++kq)
+                                umma_tf32_ss(acc + m * cfg.bn, desc_rows(a_addr + kq * 32),
+                                             umma_desc_k_sw128(wsl + kq * 32, 1024), idesc,
+                                             (kb > 0 || t > 0 || kq > 0) ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&s_wfree[rw.s]));
+                        rw.advance(cfg.n_w);
+                        if (++tj == p.kw) { tj = 0; ++ti; }
+                    }
+                    if (aborted(abort_flag)) break;
+                    umma_commit(smem_u32(&s_pfree[rp.s]));
+                    rp.advance(cfg.n_p);
+                }
+                if (aborted(abort_flag)) break;
+                umma_commit(smem_u32(&s_accfull[ab]));
+                if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
+                ab ^= 1u;
+            }
+        }
+    } else if (warp >= 4) {
+        // =========================== epilogue ===========================
+        const int q = warp & 3;
+        const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+        const int n_blk = cfg.bn / 32;
+        uint32_t ti = 0, nb = 0;   // items done, staging buffers filled
+        for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
+            const ItemPos it = item_of(work, cfg);
+            const int ab = static_cast<int>(ti & 1u);
+            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
+            if (!ok) *abort_flag = 8;
+            if (epi_bar_or(!ok || aborted(abort_flag))) break;   // all four warps leave together or not at all
+            tc_fence_after();
+            const int o0 = it.slice * cfg.bn;
+            for (int blk = 0; blk < n_blk; ++blk, ++nb) {
+                const uint32_t buf = staging + (nb & 1u) * cfg.stage_bytes;
+                if (tid == 128 && nb >= 2) tma_store_wait_read_n<1>();   // the stores that last read this buffer are done
+                epi_bar();
+                for (int m = 0; m < cfg.mt; ++m) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + ab * acc_cols + m * cfg.bn + blk * 32, v);
+                    tmem_ld_wait();
+                    if (blk == n_blk - 1 && m == cfg.mt - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+                    }
+                    const int pos = m * BM + q * 32 + lane;
+                    const int r = pos / cfg.wp, ow = pos - r * cfg.wp;
+                    if (r < cfg.r_rows) {
+                        const int srow = r * cfg.wp8 + ow;
+                        const uint32_t row_addr = buf + static_cast<uint32_t>(srow) * 128u;
+                        const uint32_t rx = static_cast<uint32_t>(srow & 7);
+#pragma unroll
+                        for (int qq = 0; qq < 8; ++qq) {
+                            float o[4];
+                            float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
+                            o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
+                            o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
+                            o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
+                            o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
+                            if (p.relu) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
+                            }
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((qq ^ rx) << 4)),
+                                         "f"(o[0]), "f"(o[1]), "f"(o[2]), "f"(o[3])
+                                         : "memory");
+                        }
+                    }
+                }
+                fence_proxy_async();
+                epi_bar();
+                if (tid == 128) {
+                    for (int r = 0; r < cfg.r_rows; ++r)
+                        if (it.oh0 + r < p.ho)
+                            tma_store_4d(&tm_y, buf + static_cast<uint32_t>(r * cfg.wp8) * 128u, o0 + blk * 32, 0, it.oh0 + r, it.n);
+                    tma_store_commit();
+                }
+            }
+        }
+        if (tid == 128) tma_store_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && s_abort != 0) {
+        atomicExch(p.status + 0, static_cast<int>(NM_ERR_TIMEOUT));
+        atomicExch(p.status + 1, 60 + s_abort);
+        atomicExch(p.status + 2, static_cast<int>(blockIdx.x));
+    }
+    if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            n = 148;
+    }
+    return n;
+}
+
+bool make_cfg(const ConvParams& p, const nm_plan_t* plan, WinCfg* cfg, size_t* smem_out)
+{
+    if (!p.wx || !nmtm::available()) return false;
+    if (p.stride_h != 1 || p.stride_w != 1 || p.kh * p.kw < 2) return false;
+    if (p.c_in % 32 != 0 || p.c_out % 32 != 0) return false;
+    if (p.pad_w > 127 || p.pad_h > 127) return false;
+    const int wp = p.w + 2 * p.pad_w;
+    if (wp - p.dil_w * (p.kw - 1) != p.wo || p.wo > 256) return false;
+    int mt = plan && plan->split > 0 ? plan->split : (wp > BM ? 2 : 1);
+    if (mt < 1 || mt > 2 || wp > BM * mt) return false;
+    int r_rows = (BM * mt) / wp;
+    if (r_rows > p.ho) r_rows = p.ho;
+    const int pr = r_rows + (p.kh - 1) * p.dil_h;
+    if (pr > 256 || wp > 256) return false;
+    int bn = 0;
+    if (plan && plan->bn > 0) {
+        bn = plan->bn;
+    } else {
+        for (int cand : {256, 128, 64, 32, 96, 160, 192, 224})
+            if (cand <= p.c_out && p.c_out % cand == 0 && 2 * mt * cand <= 512) { bn = cand; break; }
+    }
+    if (bn < 32 || bn > 256 || bn % 32 != 0 || p.c_out % bn != 0 || 2 * mt * bn > 512) return false;
+    cfg->bn = bn;
+    cfg->n_slices = p.c_out / bn;
+    cfg->mt = mt;
+    cfg->r_rows = r_rows;
+    cfg->wp = wp;
+    cfg->wp8 = (wp + 7) / 8 * 8;
+    cfg->pr = pr;
+    cfg->patch_bytes = pr * wp * 128;
+    if (cfg->patch_bytes >= (1 << 20)) return false;
+    // rows the last M-tile's furthest tap can touch: junk positions read past the patch proper
+    int rows = BM * mt + (p.kh - 1) * p.dil_h * wp + (p.kw - 1) * p.dil_w;
+    if (rows < pr * wp) rows = pr * wp;
+    cfg->pslot_bytes = ((rows * 128 + 1023) / 1024) * 1024;
+    cfg->n_kb = p.c_in / 32;
+    cfg->row_blocks = (p.ho + r_rows - 1) / r_rows;
+    cfg->stage_bytes = r_rows * cfg->wp8 * 128;
+    cfg->n_work = static_cast<long long>(p.batch) * cfg->row_blocks * cfg->n_slices;
+    const int wslot = ((bn * 128 + 1023) / 1024) * 1024;
+    const int budget = 227 * 1024 - 2048 - 2 * cfg->stage_bytes;
+    int n_p = 2, n_w = plan && plan->stages > 0 ? plan->stages : MAX_W;
+    if (n_w > MAX_W || n_w < 2) return false;
+    while (n_w > 3 && n_p * cfg->pslot_bytes + n_w * wslot > budget) --n_w;
+    if (n_p * cfg->pslot_bytes + n_w * wslot > budget) return false;
+    while (n_p < MAX_P && (n_p + 1) * cfg->pslot_bytes + n_w * wslot <= budget) ++n_p;
+    cfg->n_p = n_p;
+    cfg->n_w = n_w;
+    size_t smem = 1024 + static_cast<size_t>(n_p) * cfg->pslot_bytes + static_cast<size_t>(n_w) * wslot + 2 * cfg->stage_bytes;
+    *smem_out = smem < 120 * 1024 ? 120 * 1024 : smem;
+    return true;
+}
+
+// Activations as a tiled map (C, W, H, N) with a 32-channel x Wp x PR x 1 box: rows and columns
+// outside the image (the padding) are filled with zeros by the load.
+bool encode_x_patch(const ConvParams& p, const WinCfg& cfg, CUtensorMap* tm)
+{
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.c_in), static_cast<cuuint64_t>(p.w), static_cast<cuuint64_t>(p.h),
+                                static_cast<cuuint64_t>(p.batch)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(p.c_in) * 4, static_cast<cuuint64_t>(p.w) * p.c_in * 4,
+                                   static_cast<cuuint64_t>(p.h) * p.w * p.c_in * 4};
+    const cuuint32_t box[4] = {32, static_cast<cuuint32_t>(cfg.wp), static_cast<cuuint32_t>(cfg.pr), 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    return nmtm::encoders().tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(p.x), dims, strides, box, es,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Output as (C_out, Wo, Ho, N) with a 32-channel x Wo x 1 x 1 box: one output row per store.
+bool encode_y_row(const ConvParams& p, CUtensorMap* tm)
+{
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.c_out), static_cast<cuuint64_t>(p.wo),
+                                static_cast<cuuint64_t>(p.ho), static_cast<cuuint64_t>(p.batch)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(p.c_out) * 4, static_cast<cuuint64_t>(p.wo) * p.c_out * 4,
+                                   static_cast<cuuint64_t>(p.ho) * p.wo * p.c_out * 4};
+    const cuuint32_t box[4] = {32, static_cast<cuuint32_t>(p.wo), 1, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    return nmtm::encoders().tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.y, dims, strides, box, es,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+namespace nmhost {
+
+bool window_plan_ok(const ConvParams& p, const nm_plan_t* plan)
+{
+    WinCfg cfg;
+    size_t smem;
+    return make_cfg(p, plan, &cfg, &smem);
+}
+
+nm_status_t launch_conv_window(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st)
+{
+    WinCfg cfg;
+    size_t smem = 0;
+    if (!make_cfg(p, plan, &cfg, &smem))
+        return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the window kernel does not take this layer / plan");
+    alignas(64) CUtensorMap tm_x, tm_y;
+    if (!encode_x_patch(p, cfg, &tm_x) || !encode_y_row(p, &tm_y))
+        return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 6)");
+    cudaError_t e = cudaFuncSetAttribute(k_conv_window, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 6): %s", cudaGetErrorString(e));
+    const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
+    e = launch_pdl(k_conv_window, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x, tm_y);
+    count_launch(1);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 6): %s", cudaGetErrorString(e));
+    return NM_OK;
+}
+
+}  // namespace nmhost

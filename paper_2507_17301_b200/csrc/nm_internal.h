@@ -102,6 +102,10 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
 bool rowrun_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_rowrun(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 
+// nm_conv_window.cu — variant 6
+bool window_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_window(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
 // nm_conv_stream.cu — variant 3
 bool stream_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_stream(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);

@@ -37,6 +37,11 @@ def _plans(nm, s):
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
     out.append(p)
+    # window kernel: default, one M-tile with 64 channels, two M-tiles, short weight ring
+    for bn, mt, stages in ((0, 0, 0), (64, 1, 0), (0, 2, 0), (32, 1, 3)):
+        p = nm.nm_plan_t()
+        p.variant, p.bn, p.split, p.stages = 6, bn, mt, stages
+        out.append(p)
     return out
 
 
@@ -144,6 +149,30 @@ def test_rowrun_shapes(nm, s):
 @pytest.mark.parametrize("s", ROWRUN[:4], ids=lambda s: s.name)
 def test_rowrun_shapes_integer_exact(nm, s):
     _run(nm, s, integer=True, need_variant=[5])
+
+
+# stride-1 spatial kernels with c_in and c_out multiples of 32: window kernel
+WINDOW = [
+    ConvShape("win_3x3_56", 1, 56, 56, 64, 64, 3, 3, 1, 1, 1, 2, 4, 64),
+    ConvShape("win_3x3_28", 2, 28, 28, 128, 128, 3, 3, 1, 1, 1, 2, 4, 64),
+    ConvShape("win_3x3_14", 3, 14, 14, 64, 96, 3, 3, 1, 1, 1, 2, 4, 32),              # row blocks of 8 and 6 rows
+    ConvShape("win_5x5_dil2", 1, 20, 20, 32, 32, 5, 5, 1, 4, 2, 2, 4, 16),
+    ConvShape("win_nopad", 1, 18, 18, 32, 64, 3, 3, 1, 0, 1, 1, 4, 64),
+    ConvShape("win_wide_122", 1, 6, 120, 32, 32, 3, 3, 1, 1, 1, 2, 4, 32),            # one output row per M-tile
+    ConvShape("win_wide_132", 1, 6, 130, 32, 32, 3, 3, 1, 1, 1, 2, 4, 32),            # an output row spans two M-tiles
+    ConvShape("win_7x7_map", 4, 7, 7, 64, 64, 3, 3, 1, 1, 1, 2, 4, 64),
+    ConvShape("win_many_items", 6, 56, 56, 32, 64, 3, 3, 1, 1, 1, 2, 4, 32),          # 168+ work items: several per CTA
+]
+
+
+@pytest.mark.parametrize("s", WINDOW, ids=lambda s: s.name)
+def test_window_shapes(nm, s):
+    _run(nm, s, need_variant=[6])
+
+
+@pytest.mark.parametrize("s", WINDOW[:5] + WINDOW[6:7], ids=lambda s: s.name)
+def test_window_shapes_integer_exact(nm, s):
+    _run(nm, s, integer=True, need_variant=[6])
 
 
 @pytest.mark.parametrize("s", MEDIUM, ids=lambda s: s.name)
