@@ -291,6 +291,7 @@ def main():
     ap.add_argument("--variant", type=int, default=None, help="force a kernel variant instead of auto-tuning")
     ap.add_argument("--bn", type=int, default=0, help="with --variant: output channels per CTA")
     ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
+    ap.add_argument("--split", type=int, default=0, help="with --variant: the plan's split field")
     ap.add_argument("--save-plans", default=None, help="write the auto-tuned plans to this JSON file")
     ap.add_argument("--load-plans", default=None, help="use the plans of this JSON file instead of auto-tuning")
     args = ap.parse_args()
@@ -335,7 +336,7 @@ def main():
             plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
         else:
             plan = nm.nm_plan_t()
-            plan.variant, plan.bn, plan.stages = args.variant, args.bn, args.stages
+            plan.variant, plan.bn, plan.stages, plan.split = args.variant, args.bn, args.stages, args.split
         state.append((s, hnd, x, bias, y, plan))
 
     if args.save_plans and rank == 0:

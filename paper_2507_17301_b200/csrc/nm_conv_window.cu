@@ -13,7 +13,8 @@
 //   patch producer (1 thread)   one 4-D tiled TMA load per 32-channel block and work item
 //   weight producer (1 thread)  one contiguous bulk copy per (32-channel block, tap): the
 //                               expanded, pre-swizzled weights [BN x 32] (zeros = pruned columns)
-//   MMA issuer (1 thread)       per block and tap four 128 x BN x 8 TF32 tcgen05.mma per M-tile
+//   MMA issuers (1 thread per   per block and tap four 128 x BN x 8 TF32 tcgen05.mma
+//   M-tile)
 //   epilogue (4 warps)          TMEM -> registers, + bias, ReLU, staging in output-row order, one TMA
 //                               store per output row and 32-channel block
 // A work item is (image, block of R output rows, BN channels) with R * Wp <= 128 * MT positions
@@ -122,9 +123,9 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
 
     if (warp == 2) tmem_alloc(smem_u32(&s_tmem), 512);
     if (tid == 0) {
-        for (int i = 0; i < MAX_P; ++i) { mbar_init(smem_u32(&s_pfull[i]), 1); mbar_init(smem_u32(&s_pfree[i]), 1); }
-        for (int i = 0; i < MAX_W; ++i) { mbar_init(smem_u32(&s_wfull[i]), 1); mbar_init(smem_u32(&s_wfree[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&s_accfull[i]), 1); mbar_init(smem_u32(&s_accfree[i]), 4); }
+        for (int i = 0; i < MAX_P; ++i) { mbar_init(smem_u32(&s_pfull[i]), 1); mbar_init(smem_u32(&s_pfree[i]), cfg.mt); }
+        for (int i = 0; i < MAX_W; ++i) { mbar_init(smem_u32(&s_wfull[i]), 1); mbar_init(smem_u32(&s_wfree[i]), cfg.mt); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&s_accfull[i]), cfg.mt); mbar_init(smem_u32(&s_accfree[i]), 4); }
         mbar_fence_init();
         s_abort = 0;
         tma_prefetch_desc(&tm_x);
@@ -193,37 +194,45 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp == 1) {
-        // =========================== MMA issuer ===========================
+    } else if (warp == 1 || (warp == 2 && cfg.mt == 2)) {
+        // =========================== MMA issuers ===========================
+        // One thread per M-tile: a single thread cannot issue small MMAs as fast as the tensor core
+        // retires them, and the M-tiles have separate accumulators, so each gets its own issuer.
+        // Ring slots and accumulator hand-offs count one commit per issuer.
         if (lane == 0) {
+            const int mi = warp - 1;
             const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
+            // one tap to the right = dil_w patch rows of 128 bytes; after the last tap of a kernel row,
+            // back to the first column and dil_h patch lines (Wp rows each) down
+            const uint32_t dw_units = static_cast<uint32_t>(p.dil_w) * 8u;
+            const uint32_t dh_units = static_cast<uint32_t>(p.dil_h * cfg.wp - p.kw * p.dil_w) * 8u;
             RingPos rp, rw;
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
                 if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
                 tc_fence_after();
-                const uint32_t acc = tmem + ab * acc_cols;
+                const uint32_t acc = tmem + ab * acc_cols + mi * cfg.bn;
                 for (int kb = 0; kb < cfg.n_kb && !aborted(abort_flag); ++kb) {
                     if (!mbar_wait(smem_u32(&s_pfull[rp.s]), rp.parity)) { *abort_flag = 6; break; }
-                    const uint32_t patch = p_ring + rp.s * cfg.pslot_bytes;
-                    int ti = 0, tj = 0;
+                    // descriptors are built once per patch / weight slot and advanced by adding 16-byte units:
+                    // this thread's instruction stream is the issue rate of the whole CTA
+                    const uint64_t a_patch = desc_rows(p_ring + rp.s * cfg.pslot_bytes + mi * (BM * 128));
+                    uint32_t row_units = 0;          // (tap row offset * 128 bytes) / 16
+                    int tj = 0;
                     for (int t = 0; t < n_taps; ++t) {
                         if (!mbar_wait(smem_u32(&s_wfull[rw.s]), rw.parity)) { *abort_flag = 7; break; }
                         tc_fence_after();
-                        const uint32_t wsl = w_ring + rw.s * wslot_bytes;
-                        const uint32_t rowoff = static_cast<uint32_t>(ti * p.dil_h * cfg.wp + tj * p.dil_w) * 128u;
-                        for (int m = 0; m < cfg.mt; ++m) {
-                            const uint32_t a_addr = patch + static_cast<uint32_t>(m) * (BM * 128u) + rowoff;
-#pragma unroll
-                            for (int kq = 0; kq < 4; ++kq)
-                                umma_tf32_ss(acc + m * cfg.bn, desc_rows(a_addr + kq * 32),
-                                             umma_desc_k_sw128(wsl + kq * 32, 1024), idesc,
-                                             (kb > 0 || t > 0 || kq > 0) ? 1u : 0u);
-                        }
+                        const uint64_t b_desc = umma_desc_k_sw128(w_ring + rw.s * wslot_bytes, 1024);
+                        const uint64_t a_desc = a_patch + row_units;
+                        umma_tf32_ss(acc, a_desc, b_desc, idesc, (kb > 0 || t > 0) ? 1u : 0u);
+                        umma_tf32_ss(acc, a_desc + 2, b_desc + 2, idesc, 1u);
+                        umma_tf32_ss(acc, a_desc + 4, b_desc + 4, idesc, 1u);
+                        umma_tf32_ss(acc, a_desc + 6, b_desc + 6, idesc, 1u);
                         umma_commit(smem_u32(&s_wfree[rw.s]));
                         rw.advance(cfg.n_w);
-                        if (++tj == p.kw) { tj = 0; ++ti; }
+                        row_units += dw_units;
+                        if (++tj == p.kw) { tj = 0; row_units += dh_units; }
                     }
                     if (aborted(abort_flag)) break;
                     umma_commit(smem_u32(&s_pfree[rp.s]));
