@@ -124,7 +124,7 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
             int issued = 0;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
                 const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
-                if (rs.wrapped && !mbar_wait(smem_u32(&s_rfree[rs.s]), rs.parity ^ 1u)) { *abort_flag = 2; break; }
+                if (rs.wrapped && !mbar_wait_lone(smem_u32(&s_rfree[rs.s]), rs.parity ^ 1u)) { *abort_flag = 2; break; }
                 const int ih0 = oh * p.stride_h - p.pad_h;
                 const uint32_t bar = smem_u32(&s_rfull[rs.s]);
                 const uint32_t dst0 = rowbuf + rs.s * cfg.rowset_bytes;
@@ -173,11 +173,11 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-                if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
+                if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
                 for (int j = 0; j < cfg.nkb; ++j) {
-                    if (!mbar_wait(smem_u32(&s_afull[rp.s]), rp.parity)) { *abort_flag = 6; break; }
+                    if (!mbar_wait_lone(smem_u32(&s_afull[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     tc_fence_after();
                     const uint64_t adesc = umma_desc_k_sw128(a_ring + rp.s * SUB_BYTES, 1024);
                     const uint64_t bdesc = umma_desc_k_sw128(w_smem + j * cfg.bn * 128, 1024);

@@ -177,7 +177,7 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                 const uint8_t* rsrc = p.rel2 + static_cast<size_t>(slice * g) * rpitch;
                 int ch = 0, off_w = 0, off_h = 0, tw = 0, k0 = 0;   // position of the next 32-column sub-tile
                 for (int c = 0; c < n_chunks; ++c) {
-                    if (rp.wrapped && !mbar_wait(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
+                    if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
                     const uint32_t b_smem = ring + rp.s * cfg.stage_bytes;
                     const uint32_t slab = b_smem + cfg.b_bytes;
@@ -221,15 +221,15 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
             uint32_t ab = 0, acc_par = 0;           // accumulator buffer of this item, parity of its current use
             bool acc_wrapped = false;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-                if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
+                if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
                     *abort_flag = 5;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
                 for (int c = 0; c < n_chunks; ++c) {
-                    if (!mbar_wait(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
-                    if (!mbar_wait(smem_u32(&s_aready[set]), set_par)) { *abort_flag = 7; break; }
+                    if (!mbar_wait_lone(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
+                    if (!mbar_wait_lone(smem_u32(&s_aready[set]), set_par)) { *abort_flag = 7; break; }
                     if (aborted(abort_flag)) break;
                     tc_fence_after();
                     const uint32_t b_smem = ring + rp.s * cfg.stage_bytes;

@@ -146,7 +146,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
                 const ItemPos it = item_of(work, cfg);
                 for (int kb = 0; kb < cfg.n_kb; ++kb) {
-                    if (rp.wrapped && !mbar_wait(smem_u32(&s_pfree[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
+                    if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_pfree[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
                     const uint32_t bar = smem_u32(&s_pfull[rp.s]);
                     mbar_arrive_expect_tx(bar, static_cast<uint32_t>(cfg.patch_bytes));
@@ -175,7 +175,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
                 for (int kb = 0; kb < cfg.n_kb && !aborted(abort_flag); ++kb) {
                     const float* wsrc = w0 + static_cast<size_t>(kb) * blk_floats;   // tap 0 of this channel block
                     for (int t = 0; t < n_taps; ++t) {
-                        if (rw.wrapped && !mbar_wait(smem_u32(&s_wfree[rw.s]), rw.parity ^ 1u)) *abort_flag = 9;
+                        if (rw.wrapped && !mbar_wait_lone(smem_u32(&s_wfree[rw.s]), rw.parity ^ 1u)) *abort_flag = 9;
                         if (aborted(abort_flag)) break;
                         const uint32_t bar = smem_u32(&s_wfull[rw.s]);
                         mbar_arrive_expect_tx(bar, w_bytes);
@@ -210,18 +210,18 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
             for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-                if (acc_wrapped && !mbar_wait(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
+                if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * acc_cols + mi * cfg.bn;
                 for (int kb = 0; kb < cfg.n_kb && !aborted(abort_flag); ++kb) {
-                    if (!mbar_wait(smem_u32(&s_pfull[rp.s]), rp.parity)) { *abort_flag = 6; break; }
+                    if (!mbar_wait_lone(smem_u32(&s_pfull[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     // descriptors are built once per patch / weight slot and advanced by adding 16-byte units:
                     // this thread's instruction stream is the issue rate of the whole CTA
                     const uint64_t a_patch = desc_rows(p_ring + rp.s * cfg.pslot_bytes + mi * (BM * 128));
                     uint32_t row_units = 0;          // (tap row offset * 128 bytes) / 16
                     int tj = 0;
                     for (int t = 0; t < n_taps; ++t) {
-                        if (!mbar_wait(smem_u32(&s_wfull[rw.s]), rw.parity)) { *abort_flag = 7; break; }
+                        if (!mbar_wait_lone(smem_u32(&s_wfull[rw.s]), rw.parity)) { *abort_flag = 7; break; }
                         tc_fence_after();
                         const uint64_t b_desc = umma_desc_k_sw128(w_ring + rw.s * wslot_bytes, 1024);
                         const uint64_t a_desc = a_patch + row_units;

@@ -57,6 +57,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait: about a second at worst, then gives up and reports false.
 constexpr uint32_t kWaitPolls = 1u << 22;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
@@ -83,6 +97,15 @@ struct RingPos {
         }
     }
 };
+
+// Wait of a lone producer / issuer thread: a non-blocking test first (it returns in less than half
+// the time of the blocking form when the phase is already complete, which is the common case in a
+// full pipeline), then the bounded blocking wait.  Not for whole warps: many lanes spinning on
+// test_wait load the barrier unit.
+__device__ __forceinline__ bool mbar_wait_lone(uint32_t bar, uint32_t parity)
+{
+    return mbar_test_wait(bar, parity) || mbar_wait(bar, parity);
+}
 
 // ---- cp.async -----------------------------------------------------------------------------------
 // 16-byte copy; src_bytes = 0 writes zeros (used for padding taps and rows past the end).
