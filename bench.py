@@ -455,6 +455,34 @@ def main():
             "note": "algorithmic bytes of the layers this kernel runs / their summed launch times (median of 5 per layer)",
         }
 
+        # the same stack restricted to the kernels that gather only the retained columns (variants 1-3:
+        # Algorithm 1 proper, kept FLOPs only); the headline lets the auto-tuner also take the
+        # expanded-operand kernels, which multiply the zeros
+        if args.variant is None and not args.load_plans and not args.layer:
+            os.environ["NM_AUTOTUNE_VARIANTS"] = "1,2,3"
+            gplans = []
+            for s, hnd, x, bias, y, plan in state:
+                gp, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
+                gplans.append(gp)
+            del os.environ["NM_AUTOTUNE_VARIANTS"]
+
+            def gather_step():
+                for (s, hnd, x, bias, y, plan), gp in zip(state, gplans):
+                    nm.nm_conv2d(hnd, x, s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=y, plan=gp)
+            for _ in range(3):
+                gather_step()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+            a.record()
+            for _ in range(args.steps):
+                gather_step()
+            b.record()
+            b.synchronize()
+            g_ms = a.elapsed_time(b) / args.steps
+            out["gather_only"] = {"value": args.batch / (g_ms * 1e-3), "unit": UNIT, "ms_per_step": g_ms,
+                                  "useful_tflops": flops_step / (g_ms * 1e-3) / 1e12,
+                                  "note": "plans restricted to the gathering kernels (variants 1-3)"}
+
         # cuDNN dense convolution on the same shapes (context, unpruned weights, TF32 allowed)
         try:
             torch.backends.cudnn.allow_tf32 = True

@@ -212,6 +212,8 @@ nm_status_t nm_conv2d_host(const nm_weights_t* w, const float* x_host, float* x_
  * several), writes the fastest to *best and its time to *best_ms (may be NULL).  x and y_scratch
  * are caller buffers of the sizes nm_conv2d expects; y_scratch is overwritten.  Synchronises the
  * stream.  A candidate that fails to launch is skipped; NM_ERR_UNSUPPORTED if none runs.
+ * The environment variable NM_AUTOTUNE_VARIANTS (a list of variant digits such as "1,2,3") restricts the
+ * search, e.g. to the kernels that skip the pruned columns.
  */
 nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h, int wd,
                         int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,

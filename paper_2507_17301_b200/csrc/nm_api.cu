@@ -184,6 +184,14 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     std::memset(&a, 0, sizeof(a));
     a.variant = 1;
     out.push_back(a);
+    // NM_AUTOTUNE_VARIANTS="1,2,3" restricts the search (e.g. to the kernels that gather only the
+    // retained columns); unset = every variant
+    if (const char* allow = std::getenv("NM_AUTOTUNE_VARIANTS")) {
+        std::vector<nm_plan_t> kept;
+        for (const nm_plan_t& c : out)
+            if (std::strchr(allow, '0' + c.variant)) kept.push_back(c);
+        if (!kept.empty()) out.swap(kept);
+    }
     return out;
 }
 

@@ -255,12 +255,12 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
             const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
             const int ih0 = oh * p.stride_h - p.pad_h;
-            bool ok = mbar_wait(smem_u32(&s_rfull[rs.s]), rs.parity);
+            bool ok = mbar_wait_lone(smem_u32(&s_rfull[rs.s]), rs.parity);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 3;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             const uint32_t rows = rowbuf + rs.s * cfg.rowset_bytes;
             for (int j = 0; j < cfg.nkb; ++j) {
-                ok = !rp.wrapped || mbar_wait(smem_u32(&s_afree[rp.s]), rp.parity ^ 1u);
+                ok = !rp.wrapped || mbar_wait_lone(smem_u32(&s_afree[rp.s]), rp.parity ^ 1u);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
                 if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
                 const int ko = s_koff[j * 32 + lane];

@@ -332,9 +332,9 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
         for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
             for (int c = 0; c < n_chunks; ++c) {
                 const int s = rp.s;
-                bool ok = mbar_wait(smem_u32(&s_full[s]), rp.parity);
+                bool ok = mbar_wait_lone(smem_u32(&s_full[s]), rp.parity);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 3;
-                ok = !set_wrapped || mbar_wait(smem_u32(&s_afree[set]), set_par ^ 1u);
+                ok = !set_wrapped || mbar_wait_lone(smem_u32(&s_afree[set]), set_par ^ 1u);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
                 if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
                 tc_fence_after();

@@ -98,9 +98,9 @@ struct RingPos {
     }
 };
 
-// Wait of a lone producer / issuer thread: a non-blocking test first (it returns in less than half
-// the time of the blocking form when the phase is already complete, which is the common case in a
-// full pipeline), then the bounded blocking wait.  Not for whole warps: many lanes spinning on
+// Wait that is usually already satisfied (a stage of a full pipeline): one non-blocking test first
+// (it returns in less than half the time of the blocking form when the phase is complete), then
+// the bounded blocking wait.  The test is made once, not in a loop: many lanes spinning on
 // test_wait load the barrier unit.
 __device__ __forceinline__ bool mbar_wait_lone(uint32_t bar, uint32_t parity)
 {
