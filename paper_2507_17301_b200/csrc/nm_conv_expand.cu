@@ -57,6 +57,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t n_work = static_cast<uint32_t>(cfg.n_work);   // below 2^31: per-item arithmetic stays 32-bit
     const int NS = cfg.stages, n_sub = cfg.n_sub;
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t staging = ring + NS * cfg.stage_bytes;
@@ -93,11 +94,11 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
             const size_t w_step = static_cast<size_t>(p.c_out) * 32;   // floats between two 32-column blocks
             RingPos rp;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-                const int slice = static_cast<int>(work % cfg.n_slices);
-                const long long pix0 = (work / cfg.n_slices) * BM;
-                const int n0 = static_cast<int>(pix0 / hw);
-                const int rem = static_cast<int>(pix0 - static_cast<long long>(n0) * hw);
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
+                const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
+                const uint32_t pix0 = (work / static_cast<uint32_t>(cfg.n_slices)) * BM;
+                const int n0 = static_cast<int>(pix0 / static_cast<uint32_t>(hw));
+                const int rem = static_cast<int>(pix0 - static_cast<uint32_t>(n0) * static_cast<uint32_t>(hw));
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
                 const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32;
@@ -138,7 +139,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             RingPos rp;
             uint32_t ab = 0, acc_par = 0;   // accumulator buffer of this item, parity of its current use
             bool acc_wrapped = false;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
                     *abort_flag = 5;
                     break;
@@ -173,9 +174,9 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t nb = 0, ti = 0;
-        for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
-            const int slice = static_cast<int>(work % cfg.n_slices);
-            const long long pix0 = (work / cfg.n_slices) * BM;
+        for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
+            const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
+            const uint32_t pix0 = (work / static_cast<uint32_t>(cfg.n_slices)) * BM;
             const int ab = static_cast<int>(ti & 1u);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
@@ -288,6 +289,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     }
     cfg->stages = stages;
     cfg->n_work = ((p.pixels + BM - 1) / BM) * cfg->n_slices;
+    if (cfg->n_work >= (1ll << 31)) return false;
     return true;
 }
 

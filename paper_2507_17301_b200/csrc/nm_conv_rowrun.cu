@@ -7,7 +7,7 @@
 //   producer (1 thread)    bulk-copies the kh input rows the item needs into shared memory: with
 //                          dil_h = 1 they are adjacent in memory, so ONE copy brings them all (rows
 //                          outside the image are simply not copied);
-//   builders (8 warps)     lay the patch matrix [128 pixels x K] down in 32-column sub-tiles in the
+//   builders (2 x 8 warps)    lay the patch matrix [128 pixels x K] down in 32-column sub-tiles in the
 //                          K-major, 128-byte-swizzled layout the tensor core reads: lane = column,
 //                          so a warp reads 32 consecutive floats of a run and writes one 128-byte
 //                          row, both free of bank conflicts.  Padding is resolved per column with a
@@ -34,7 +34,8 @@ constexpr int BM = 128;
 constexpr int SUB_BYTES = BM * 128;
 constexpr int A_RING = 4;
 constexpr int MAX_SETS = 4;   // row sets in flight: the copy of item i + n_sets - 1 is issued while item i is built
-constexpr int THREADS = 512;
+constexpr int NB_GROUPS = 2;                  // builder groups of 8 warps taking alternate sub-tiles
+constexpr int THREADS = (8 + 8 * NB_GROUPS) * 32;
 constexpr int STAGING_BYTES = 4 * 2 * 4096;
 constexpr int MAX_KB = 16;   // sub-tiles of 32 columns: K <= 512
 
@@ -63,6 +64,7 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
     __shared__ uint32_t s_range[MAX_KB * 32];   // per column: first valid output pixel << 16 | number of valid ones
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t n_work = static_cast<uint32_t>(cfg.n_work);   // below 2^31: per-item arithmetic stays 32-bit
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t w_smem = base;
     const uint32_t a_ring = w_smem + ((cfg.w_bytes + 1023) / 1024) * 1024;
@@ -76,7 +78,7 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         mbar_init(smem_u32(&s_wfull), 1);
         for (int i = 0; i < MAX_SETS; ++i) {
             mbar_init(smem_u32(&s_rfull[i]), 1);
-            mbar_init(smem_u32(&s_rfree[i]), 8);
+            mbar_init(smem_u32(&s_rfree[i]), 8 * NB_GROUPS);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&s_accfull[i]), 1);
@@ -122,8 +124,8 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
             bulk_load_1d(w_smem, p.wx, static_cast<uint32_t>(cfg.w_bytes), smem_u32(&s_wfull));
             RingPos rs;
             int issued = 0;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-                const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
+                const int n = static_cast<int>(work / static_cast<uint32_t>(p.ho)), oh = static_cast<int>(work - static_cast<uint32_t>(n) * static_cast<uint32_t>(p.ho));
                 if (rs.wrapped && !mbar_wait_lone(smem_u32(&s_rfree[rs.s]), rs.parity ^ 1u)) { *abort_flag = 2; break; }
                 const int ih0 = oh * p.stride_h - p.pad_h;
                 const uint32_t bar = smem_u32(&s_rfull[rs.s]);
@@ -172,7 +174,7 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
             RingPos rp;
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
@@ -201,7 +203,7 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t nb = 0, ti = 0;
-        for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
+        for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
             const int ab = static_cast<int>(ti & 1u);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
@@ -249,17 +251,25 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
         if (lane == 0) tma_store_wait_all();
     } else if (warp >= 8) {
         // =========================== builders ===========================
-        const int bw = warp - 8;   // rows bw, bw + 8, ...
+        // Two groups of eight warps build alternate sub-tiles, so that one group's barrier waits and
+        // arrivals overlap the other's loads and stores.  Inside a group warp bw takes rows bw, bw + 8, ...
+        const int bw = (warp - 8) & 7;
+        const int grp = (warp - 8) >> 3;
+        uint32_t turn = 0;   // parity of the running sub-tile count: whose sub-tile the next one is
         RingPos rp;
         RingPos rs;
-        for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-            const int n = static_cast<int>(work / p.ho), oh = static_cast<int>(work - static_cast<long long>(n) * p.ho);
+        for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
+            const int n = static_cast<int>(work / static_cast<uint32_t>(p.ho)), oh = static_cast<int>(work - static_cast<uint32_t>(n) * static_cast<uint32_t>(p.ho));
             const int ih0 = oh * p.stride_h - p.pad_h;
             bool ok = mbar_wait_lone(smem_u32(&s_rfull[rs.s]), rs.parity);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 3;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             const uint32_t rows = rowbuf + rs.s * cfg.rowset_bytes;
-            for (int j = 0; j < cfg.nkb; ++j) {
+            for (int j = 0; j < cfg.nkb; ++j, turn ^= 1u) {
+                if (turn != static_cast<uint32_t>(grp)) {   // the other group's sub-tile
+                    rp.advance(A_RING);
+                    continue;
+                }
                 ok = !rp.wrapped || mbar_wait_lone(smem_u32(&s_afree[rp.s]), rp.parity ^ 1u);
                 if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
                 if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;

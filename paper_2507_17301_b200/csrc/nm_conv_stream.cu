@@ -128,6 +128,7 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t n_work = static_cast<uint32_t>(cfg.n_work);   // below 2^31: per-item arithmetic stays 32-bit
     const int NS = cfg.stages, n_chunks = p.v2_chunks, g = cfg.g, T = p.tile_t;
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t staging = ring + NS * cfg.stage_bytes;
@@ -167,11 +168,11 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
             const uint32_t tx_fixed = static_cast<uint32_t>(cfg.bn) * 128u + static_cast<uint32_t>(g) * 32u;
             RingPos rp;
             int issued = 0;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
-                const int slice = static_cast<int>(work % cfg.n_slices);
-                const long long pix0 = (work / cfg.n_slices) * BM;
-                const int n0 = static_cast<int>(pix0 / hw);
-                const int rem = static_cast<int>(pix0 - static_cast<long long>(n0) * hw);
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
+                const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
+                const uint32_t pix0 = (work / static_cast<uint32_t>(cfg.n_slices)) * BM;
+                const int n0 = static_cast<int>(pix0 / static_cast<uint32_t>(hw));
+                const int rem = static_cast<int>(pix0 - static_cast<uint32_t>(n0) * static_cast<uint32_t>(hw));
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
                 const uint8_t* rsrc = p.rel2 + static_cast<size_t>(slice * g) * rpitch;
@@ -220,7 +221,7 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
             uint32_t set = 0, set_par = 0;          // operand set of this chunk, parity of its current use
             uint32_t ab = 0, acc_par = 0;           // accumulator buffer of this item, parity of its current use
             bool acc_wrapped = false;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
                     *abort_flag = 5;
                     break;
@@ -267,9 +268,9 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
         const int n_blk = cfg.bn / 32;
         uint32_t ti = 0;
         uint32_t nb = 0;  // staging boxes this warp has filled so far
-        for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
-            const int slice = static_cast<int>(work % cfg.n_slices);
-            const long long pix0 = (work / cfg.n_slices) * BM;
+        for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
+            const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
+            const uint32_t pix0 = (work / static_cast<uint32_t>(cfg.n_slices)) * BM;
             const int ab = cfg.n_acc == 2 ? static_cast<int>(ti & 1u) : 0;
             const bool ok = aborted(abort_flag) ||
                             mbar_wait(smem_u32(&s_accfull[ab]), (cfg.n_acc == 2 ? (ti >> 1) : ti) & 1u);
@@ -329,7 +330,7 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
         RingPos rp;
         uint32_t set = 0, set_par = 0;
         bool set_wrapped = false;
-        for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+        for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
             for (int c = 0; c < n_chunks; ++c) {
                 const int s = rp.s;
                 bool ok = mbar_wait_lone(smem_u32(&s_full[s]), rp.parity);
@@ -478,6 +479,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, StreamCfg* cfg)
     cfg->stages = stages;
     const long long pix_blocks = (p.pixels + BM - 1) / BM;
     cfg->n_work = pix_blocks * cfg->n_slices;
+    if (cfg->n_work >= (1ll << 31)) return false;
     return true;
 }
 

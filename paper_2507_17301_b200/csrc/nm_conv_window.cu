@@ -90,13 +90,13 @@ __device__ __forceinline__ uint64_t desc_rows(uint32_t addr) { return umma_desc_
 struct ItemPos {
     int slice, n, oh0;
 };
-__device__ __forceinline__ ItemPos item_of(long long work, const WinCfg& cfg)
+__device__ __forceinline__ ItemPos item_of(uint32_t work, const WinCfg& cfg)
 {
     ItemPos it;
-    it.slice = static_cast<int>(work % cfg.n_slices);
-    const long long rest = work / cfg.n_slices;
-    const int rb = static_cast<int>(rest % cfg.row_blocks);
-    it.n = static_cast<int>(rest / cfg.row_blocks);
+    it.slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
+    const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
+    const int rb = static_cast<int>(rest % static_cast<uint32_t>(cfg.row_blocks));
+    it.n = static_cast<int>(rest / static_cast<uint32_t>(cfg.row_blocks));
     it.oh0 = rb * cfg.r_rows;
     return it;
 }
@@ -111,6 +111,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t n_work = static_cast<uint32_t>(cfg.n_work);   // below 2^31: per-item arithmetic stays 32-bit
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t p_ring = base;
     const uint32_t w_ring = p_ring + cfg.n_p * cfg.pslot_bytes;
@@ -143,7 +144,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
         if (lane == 0) {
             RingPos rp;
             int issued = 0;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 const ItemPos it = item_of(work, cfg);
                 for (int kb = 0; kb < cfg.n_kb; ++kb) {
                     if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_pfree[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
@@ -169,7 +170,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
             RingPos rw;
             int issued = 0;
             const size_t blk_floats = static_cast<size_t>(p.c_out) * 32;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 const ItemPos it = item_of(work, cfg);
                 const float* w0 = p.wx + static_cast<size_t>(it.slice) * cfg.bn * 32;
                 for (int kb = 0; kb < cfg.n_kb && !aborted(abort_flag); ++kb) {
@@ -209,7 +210,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
             RingPos rp, rw;
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
-            for (long long work = blockIdx.x; work < cfg.n_work && !aborted(abort_flag); work += gridDim.x) {
+            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) { *abort_flag = 5; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * acc_cols + mi * cfg.bn;
@@ -250,7 +251,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const int n_blk = cfg.bn / 32;
         uint32_t ti = 0, nb = 0;   // items done, staging buffers filled
-        for (long long work = blockIdx.x; work < cfg.n_work; work += gridDim.x, ++ti) {
+        for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
             const ItemPos it = item_of(work, cfg);
             const int ab = static_cast<int>(ti & 1u);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
@@ -372,6 +373,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, WinCfg* cfg, size_t* s
     cfg->row_blocks = (p.ho + r_rows - 1) / r_rows;
     cfg->stage_bytes = r_rows * cfg->wp8 * 128;
     cfg->n_work = static_cast<long long>(p.batch) * cfg->row_blocks * cfg->n_slices;
+    if (cfg->n_work >= (1ll << 31)) return false;
     const int wslot = ((bn * 128 + 1023) / 1024) * 1024;
     const int budget = 227 * 1024 - 2048 - 2 * cfg->stage_bytes;
     int n_p = 2, n_w = plan && plan->stages > 0 ? plan->stages : MAX_W;
