@@ -34,6 +34,7 @@ void free_handle_memory(nm_weights* h)
     cudaFree(h->wt2);
     cudaFree(h->rel2);
     cudaFree(h->wx);
+    cudaFree(h->splitk);
     h->magic = 0;
     delete h;
 }
@@ -120,6 +121,8 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     p->rel2 = w->v2_ok ? w->rel2 : nullptr;
     p->v2_kc = w->v2_kc; p->v2_s = w->v2_s; p->v2_chunks = w->v2_chunks;
     p->wx = w->wx;
+    p->splitk = w->splitk;
+    p->splitk_bytes = w->splitk_bytes;
     return NM_OK;
 }
 
@@ -166,8 +169,14 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, &a)) out.push_back(a);
     std::memset(&a, 0, sizeof(a));
     for (int bn : {64, 128, 256}) {         // expanded-operand kernel
-        a.variant = 4; a.bn = bn; a.stages = 0;
+        a.variant = 4; a.bn = bn; a.stages = 0; a.split = 0;
         if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);
+    }
+    for (int splits : {2, 3, 4}) {          // ... with the reduction axis split (needs the handle's scratch)
+        for (int bn : {128, 256}) {
+            a.variant = 4; a.bn = bn; a.stages = 0; a.split = splits;
+            if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);
+        }
     }
     std::memset(&a, 0, sizeof(a));
     for (int bn : {0, 256, p.tile_t}) {     // stream kernel: default width, widest, one tile per CTA
@@ -354,6 +363,27 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
                                 bias, relu, y_scratch, &p);
     if (s != NM_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // Layers with fewer work items than SMs and a long reduction axis are also tried with the axis
+    // split over several CTAs; the partial sums need scratch memory, which belongs to the handle
+    // and is reserved here (nm_conv2d itself never allocates).
+    {
+        nm_weights* hw = const_cast<nm_weights*>(w);
+        int n_sm = 148, dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        const long long pix_blocks = (p.pixels + 127) / 128;
+        const bool few_items = pix_blocks * ((p.c_out + 255) / 256) < n_sm && p.k / 32 >= 32;
+        const size_t need = few_items && p.wx ? nmhost::expand_splitk_bytes(p, 4) : 0;
+        if (need > hw->splitk_bytes) {
+            cudaStreamSynchronize(st);
+            cudaFree(hw->splitk);
+            hw->splitk = nullptr;
+            hw->splitk_bytes = 0;
+            if (cudaMalloc(&hw->splitk, need) == cudaSuccess) hw->splitk_bytes = need;
+            else (void)cudaGetLastError();   // no scratch: the split plans are simply not candidates
+        }
+        p.splitk = hw->splitk;
+        p.splitk_bytes = hw->splitk_bytes;
+    }
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
         if (e0) cudaEventDestroy(e0);

@@ -40,7 +40,9 @@ struct ExpandCfg {
     int stages;
     int b_bytes;      // weight bytes per stage (bn rows of 128 bytes)
     int stage_bytes;
-    int n_sub;        // K / 32
+    int n_sub;        // 32-column blocks one work item reduces over: (K / 32) / ksplit
+    int ksplit;       // K splits (1 = none): a work item covers one of them and stores raw partial sums
+    int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
     int boxes;        // output staging boxes per epilogue warp: 2 for short reductions, 1 when the ring needs the room
     long long n_work;
 };
@@ -96,13 +98,19 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             RingPos rp;
             for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
-                const uint32_t pix0 = (work / static_cast<uint32_t>(cfg.n_slices)) * BM;
+                const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
+                const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
+                const uint32_t pix0 = (rest / static_cast<uint32_t>(cfg.ksplit)) * BM;
                 const int n0 = static_cast<int>(pix0 / static_cast<uint32_t>(hw));
                 const int rem = static_cast<int>(pix0 - static_cast<uint32_t>(n0) * static_cast<uint32_t>(hw));
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
-                const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32;
-                int ch = 0, off_w = 0, off_h = 0, tw = 0;
+                // first 32-column block of this item's share of the reduction axis
+                const int c0 = ks * n_sub;
+                const int tap0 = (c0 * 32) / p.c_in;
+                const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32 + static_cast<size_t>(c0) * w_step;
+                int ch = c0 * 32 - tap0 * p.c_in, tw = tap0 % p.kw;
+                int off_w = tw * p.dil_w, off_h = (tap0 / p.kw) * p.dil_h;
                 for (int c = 0; c < n_sub; ++c) {
                     if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
@@ -176,7 +184,9 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         uint32_t nb = 0, ti = 0;
         for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
             const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
-            const uint32_t pix0 = (work / static_cast<uint32_t>(cfg.n_slices)) * BM;
+            const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
+            const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
+            const uint32_t pix0 = (rest / static_cast<uint32_t>(cfg.ksplit)) * BM;
             const int ab = static_cast<int>(ti & 1u);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
@@ -221,7 +231,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 __syncwarp();
                 if (lane == 0) {
                     if (pix0 + q * 32 < p.pixels)
-                        tma_store_2d(&tm_y, box, o0 + blk * 32, static_cast<int>(pix0) + q * 32);
+                        tma_store_2d(&tm_y, box, o0 + blk * 32, ks * cfg.p_pad + static_cast<int>(pix0) + q * 32);
                     tma_store_commit();
                 }
             }
@@ -241,6 +251,27 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         atomicExch(p.status + 2, static_cast<int>(blockIdx.x));
     }
     if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+// Second pass of a split-K plan: y[p][c] = act(sum over splits of partial[s][p][c] + bias[c]).
+__global__ void k_splitk_reduce(const float4* __restrict__ part, int splits, size_t split_stride4, size_t n4, int c_out4,
+                                const float4* __restrict__ bias, int relu, float4* __restrict__ y)
+{
+    nmk::pdl_wait();   // the partial sums come from the kernel launched just before
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n4;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        float4 a = part[i];
+        for (int s = 1; s < splits; ++s) {
+            const float4 b = part[i + s * split_stride4];
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        if (bias) {
+            const float4 b = __ldg(bias + (i % c_out4));
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        if (relu) { a.x = fmaxf(a.x, 0.f); a.y = fmaxf(a.y, 0.f); a.z = fmaxf(a.z, 0.f); a.w = fmaxf(a.w, 0.f); }
+        y[i] = a;
+    }
 }
 
 int sm_count()
@@ -276,7 +307,14 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     cfg->n_slices = p.c_out / bn;
     cfg->b_bytes = ((bn * 128 + 1023) / 1024) * 1024;
     cfg->stage_bytes = SUB_BYTES + cfg->b_bytes;
-    cfg->n_sub = p.k / 32;
+    const int splits = plan && plan->split > 1 ? plan->split : 1;
+    if (splits > 8 || (p.k / 32) % splits != 0) return false;
+    cfg->ksplit = splits;
+    cfg->n_sub = (p.k / 32) / splits;
+    cfg->p_pad = static_cast<int>(((p.pixels + BM - 1) / BM) * BM);
+    if (splits > 1 && (!p.splitk || p.splitk_bytes < static_cast<size_t>(splits) * cfg->p_pad * p.c_out * sizeof(float) ||
+                       static_cast<long long>(splits) * cfg->p_pad >= (1ll << 31)))
+        return false;   // the partial-sum scratch is reserved by nm_autotune
     cfg->boxes = cfg->n_sub <= 8 ? 2 : 1;   // long reductions: the epilogue is rare, the ring needs the bytes
     const int budget = 227 * 1024 - 1024 - 8 * cfg->boxes * BOX_BYTES - 1024;
     int stages = plan && plan->stages > 0 ? plan->stages : NSTAGE_MAX;
@@ -288,7 +326,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
         if (stages * cfg->stage_bytes > budget) return false;
     }
     cfg->stages = stages;
-    cfg->n_work = ((p.pixels + BM - 1) / BM) * cfg->n_slices;
+    cfg->n_work = ((p.pixels + BM - 1) / BM) * cfg->n_slices * splits;
     if (cfg->n_work >= (1ll << 31)) return false;
     return true;
 }
@@ -308,19 +346,47 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     ExpandCfg cfg;
     if (!make_cfg(p, plan, &cfg))
         return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the expanded-operand kernel does not take this layer / plan");
+    // a split-K plan stores raw partial sums [split][pixel][channel] in the handle's scratch; bias and
+    // activation are applied by the reduction pass
+    ConvParams q = p;
+    if (cfg.ksplit > 1) {
+        q.y = p.splitk;
+        q.pixels = static_cast<long long>(cfg.ksplit) * cfg.p_pad;   // rows of the store map
+        q.bias = nullptr;
+        q.relu = 0;
+    }
     alignas(64) CUtensorMap tm_x, tm_y;
-    if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_y_tiled(p, &tm_y))
+    if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_y_tiled(q, &tm_y))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 4)");
+    q.pixels = p.pixels;
     size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 8 * cfg.boxes * BOX_BYTES;
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
     cudaError_t e = cudaFuncSetAttribute(k_conv_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    e = nmhost::launch_pdl(k_conv_expand, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x, tm_y);
+    e = nmhost::launch_pdl(k_conv_expand, static_cast<unsigned>(grid), THREADS, smem, st, q, cfg, tm_x, tm_y);
     nmhost::count_launch(1);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 4): %s", cudaGetErrorString(e));
+    if (cfg.ksplit > 1) {
+        const size_t n4 = static_cast<size_t>(p.pixels) * p.c_out / 4;
+        const size_t stride4 = static_cast<size_t>(cfg.p_pad) * p.c_out / 4;
+        size_t blocks = (n4 + 255) / 256;
+        if (blocks > static_cast<size_t>(sm_count()) * 8) blocks = static_cast<size_t>(sm_count()) * 8;
+        e = nmhost::launch_pdl(k_splitk_reduce, static_cast<unsigned>(blocks), 256u, 0, st,
+                               reinterpret_cast<const float4*>(p.splitk), cfg.ksplit, stride4, n4, p.c_out / 4,
+                               reinterpret_cast<const float4*>(p.bias), p.relu, reinterpret_cast<float4*>(p.y));
+        nmhost::count_launch(1);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (split-K reduction): %s", cudaGetErrorString(e));
+    }
     return NM_OK;
+}
+
+size_t expand_splitk_bytes(const ConvParams& p, int splits)
+{
+    const size_t p_pad = static_cast<size_t>((p.pixels + BM - 1) / BM) * BM;
+    return static_cast<size_t>(splits) * p_pad * p.c_out * sizeof(float);
 }
 
 }  // namespace nmhost

@@ -28,6 +28,8 @@ struct nm_weights {
     float* wt2;          // [c_out][v2_chunks * 32] TF32 weights, chunk-major, first v2_kc of each 32 used
     uint8_t* rel2;       // [n_tiles][v2_chunks * 32] source column of each kept column, relative to its chunk
     // Expanded layout (variant 4): the pruned matrix back in dense shape, zeros in the pruned columns.
+    float* splitk;       // scratch for split-K partial sums (variant 4), allocated by nm_autotune; may be NULL
+    size_t splitk_bytes;
     float* wx;           // [ceil(k / 32)][c_out][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
 };
 
@@ -52,6 +54,9 @@ struct ConvParams {
     int v2_kc, v2_s, v2_chunks;
     // expanded layout (variant 4)
     const float* wx;
+    // split-K scratch of the handle (variant 4 with plan.split > 1)
+    float* splitk;
+    size_t splitk_bytes;
 };
 
 namespace nmhost {
@@ -96,6 +101,7 @@ nm_status_t launch_conv_slab(const ConvParams& p, const nm_plan_t* plan, cudaStr
 
 // nm_conv_expand.cu — variant 4
 bool expand_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+size_t expand_splitk_bytes(const ConvParams& p, int splits);   // scratch a split-K plan of this layer needs
 nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 
 // nm_conv_rowrun.cu — variant 5

@@ -219,6 +219,40 @@ def test_small_shapes_integer_exact(nm, s):
     _run(nm, s, integer=True)
 
 
+@pytest.mark.parametrize("integer", [False, True], ids=["normal", "integer_exact"])
+def test_split_k_plans(nm, integer):
+    """Few pixel blocks and a long reduction axis: the expanded-operand kernel with the axis split over
+    2, 3 and 4 CTAs (partial sums through the handle's scratch, reserved by nm_autotune, then reduced)."""
+    s = ConvShape("splitk_3x3", 2, 14, 14, 256, 64, 3, 3, 1, 1, 1, 2, 4, 32)        # K = 2304: 72 blocks of 32
+    w, x, b = tensors_for(s, integer)
+    vr, ir, yr = oracle_layer(s, w, x, b)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    xd, bd = x.cuda(), b.cuda()
+    plan = nm.nm_plan_t()
+    plan.variant, plan.bn, plan.split = 4, 64, 2
+    with pytest.raises(nm.NmError) as e:                      # no scratch yet: the plan is refused
+        nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
+    assert e.value.status == nm.NM_ERR_UNSUPPORTED
+    best, ms = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)   # reserves the scratch
+    assert ms > 0
+    for splits in (2, 3, 4):
+        for bn in (32, 64):
+            plan = nm.nm_plan_t()
+            plan.variant, plan.bn, plan.split = 4, bn, splits
+            for _ in range(2):                                # twice: the scratch is reused
+                y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
+            nm.nm_weights_check(hnd)
+            torch.cuda.synchronize()
+            if integer:
+                assert np.array_equal(y.cpu().numpy(), yr), (splits, bn)
+            else:
+                assert_conv_close(y.cpu().numpy(), yr)
+    y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=best)
+    torch.cuda.synchronize()
+    if not integer:
+        assert_conv_close(y.cpu().numpy(), yr)
+
+
 def test_no_bias_no_relu(nm):
     _run(nm, SMALL[0].with_(relu=False), use_bias=False)
 
