@@ -38,9 +38,10 @@ UNIT = "images/s"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 TF32_OVER_BF16 = 1.1 / 2.25   # nominal dense tensor peaks: 1.1 PFLOP/s TF32, 2.25 PFLOP/s bf16
-KERNEL_OF_VARIANT = {1: "k_conv_gather", 2: "k_conv_slab", 3: "k_conv_stream", 4: "k_conv_expand", 5: "k_conv_rowrun"}
+KERNEL_OF_VARIANT = {1: "k_conv_gather", 2: "k_conv_slab", 3: "k_conv_stream", 4: "k_conv_expand", 5: "k_conv_rowrun",
+                     6: "k_conv_window"}
 KERNEL_SOURCE = {"k_conv_gather": "nm_conv_gather.cu", "k_conv_slab": "nm_conv_slab.cu", "k_conv_stream": "nm_conv_stream.cu",
-                 "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu"}
+                 "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu", "k_conv_window": "nm_conv_window.cu"}
 
 
 def peaks():
@@ -97,8 +98,15 @@ def useful_flops(s: inputs.ConvShape) -> int:
     return 2 * s.pixels * s.c_out * s.kk
 
 
+WORKLOAD = {"depth": 50, "n": 2, "m": 4, "tile": 64}   # the headline configuration; --depth / --nm / --tile change it
+
+
 def workload(batch: int):
-    return inputs.resnet_conv_stack(50, batch, 2, 4, tile_t=64)
+    return inputs.resnet_conv_stack(WORKLOAD["depth"], batch, WORKLOAD["n"], WORKLOAD["m"], tile_t=WORKLOAD["tile"])
+
+
+def workload_name(batch: int) -> str:
+    return f"resnet{WORKLOAD['depth']}_conv_stack_b{batch}_224_{WORKLOAD['n']}of{WORKLOAD['m']}"
 
 
 class ClockSampler:
@@ -243,12 +251,12 @@ def run_reference(args):
         step()
     dt = (time.perf_counter() - t0) / steps
     value = 1.0 / dt
-    sample = "image 0 of each of the 53 layers per step (1 of 64 images)"
+    sample = f"image 0 of each of the {len(layers)} layers per step (1 image of the batch)"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "resnet50_conv_stack_b64_224_2of4", "sample": sample},
+        "config": {"workload": workload_name(64), "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -274,7 +282,7 @@ def cpu_baseline(budget_s: float = 20.0):
     flops_done = sum(useful_flops(s) for s in layers[:done])
     flops_all = sum(useful_flops(s) for s in layers)
     est_image_s = t_total * flops_all / flops_done  # scaled by kept FLOPs if the budget cut the pass short
-    sample = (f"image 0 of the first {done} of 53 layers (1 of 64 images)"
+    sample = (f"image 0 of the first {done} of {len(layers)} layers (1 image of the batch)"
               + ("" if done == len(layers) else ", scaled to the stack by kept FLOPs"))
     return {"value": 1.0 / est_image_s, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample}
 
@@ -292,9 +300,13 @@ def main():
     ap.add_argument("--bn", type=int, default=0, help="with --variant: output channels per CTA")
     ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
     ap.add_argument("--split", type=int, default=0, help="with --variant: the plan's split field")
+    ap.add_argument("--depth", type=int, default=50, choices=[50, 101, 152], help="ResNet depth of the conv stack")
+    ap.add_argument("--nm", default="2:4", help="N:M pattern of the pruned layers, e.g. 1:4 or 2:8")
+    ap.add_argument("--tile", type=int, default=64, help="pruning tile width T")
     ap.add_argument("--save-plans", default=None, help="write the auto-tuned plans to this JSON file")
     ap.add_argument("--load-plans", default=None, help="use the plans of this JSON file instead of auto-tuning")
     args = ap.parse_args()
+    WORKLOAD.update(depth=args.depth, n=int(args.nm.split(":")[0]), m=int(args.nm.split(":")[1]), tile=args.tile)
     if args.impl == "reference":
         return run_reference(args)
     if args.warmup < 3:
@@ -332,6 +344,7 @@ def main():
         if loaded is not None and s.name in loaded:
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.stages, plan.split = (loaded[s.name][k] for k in ("variant", "bn", "stages", "split"))
+            nm.nm_weights_reserve(hnd, nm.nm_plan_scratch_bytes(hnd, x.shape, s.stride, s.pad, s.dil, plan))
         elif args.variant is None:
             plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
         else:
@@ -379,9 +392,9 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
         "data": "synthetic",
-        "config": {"workload": "resnet50_conv_stack_b64_224_2of4" + (f" [only {args.layer}]" if args.layer else ""),
+        "config": {"workload": workload_name(args.batch) + (f" [only {args.layer}]" if args.layer else ""),
                    "layers": len(layers), "batch_per_gpu": args.batch,
-                   "tile_t": 64, "plans": "per layer by nm_autotune" if args.variant is None and not args.load_plans else "given", "cache": "inputs larger than L2 (5.4 GB touched per step, one buffer per layer)",
+                   "tile_t": WORKLOAD["tile"], "plans": "per layer by nm_autotune" if args.variant is None and not args.load_plans else "given", "cache": f"inputs larger than L2 ({bytes_step / 1e9:.1f} GB touched per step, one buffer per layer)",
                    "parallelism": f"replicas x{world}"},
         "useful_tflops": flops_step / (ms_step * 1e-3) / 1e12,
         "gpu_launches": int(launches),

@@ -33,6 +33,7 @@
 #ifndef NM_H_
 #define NM_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -159,6 +160,20 @@ nm_status_t nm_weights_export(const nm_weights_t* w, float* values, uint16_t* in
 nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int c_out, int kh,
                               int kw, int c_in, int n_keep, int m_group, int tile_t,
                               void* cuda_stream, nm_weights_t** out);
+
+/*
+ * Scratch memory of a handle.  A plan that splits the reduction axis over several CTAs (variant 4
+ * with split > 1) passes partial sums through scratch memory owned by the handle; nm_conv2d never
+ * allocates, so the scratch must be there before such a plan is used.  nm_autotune reserves it for the
+ * layers it tunes; a caller that brings a plan from elsewhere (a plan cache) asks for the size with
+ * nm_plan_scratch_bytes (0 for plans that need none) and reserves it with nm_weights_reserve, which
+ * allocates synchronously and keeps the larger of the old and new sizes.  Calls that use the same
+ * handle's scratch must not overlap on the GPU.
+ */
+nm_status_t nm_plan_scratch_bytes(const nm_weights_t* w, int batch, int h, int wd, int stride_h, int stride_w,
+                                  int pad_h, int pad_w, int dil_h, int dil_w, const nm_plan_t* plan,
+                                  size_t* bytes);
+nm_status_t nm_weights_reserve(nm_weights_t* w, size_t bytes);
 
 /* Synchronises `cuda_stream`, then reads the handle's device status word.  Returns NM_OK, or
  * NM_ERR_TIMEOUT if a kernel that used this handle gave up on a bounded wait (the status word is

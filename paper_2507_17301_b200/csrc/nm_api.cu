@@ -291,6 +291,36 @@ nm_status_t nm_weights_export(const nm_weights_t* w, float* values, uint16_t* in
     return NM_OK;
 }
 
+nm_status_t nm_plan_scratch_bytes(const nm_weights_t* w, int batch, int h, int wd, int stride_h, int stride_w,
+                                  int pad_h, int pad_w, int dil_h, int dil_w, const nm_plan_t* plan, size_t* bytes)
+{
+    if (!bytes) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_plan_scratch_bytes: bytes is NULL");
+    *bytes = 0;
+    ConvParams p;
+    float* const dummy = reinterpret_cast<float*>(static_cast<uintptr_t>(256));   // geometry only: never dereferenced
+    nm_status_t s = make_params("nm_plan_scratch_bytes", w, dummy, batch, h, wd, stride_h, stride_w, pad_h, pad_w,
+                                dil_h, dil_w, nullptr, 0, dummy, &p);
+    if (s != NM_OK) return s;
+    if (plan && plan->variant == 4 && plan->split > 1) *bytes = nmhost::expand_splitk_bytes(p, plan->split);
+    return NM_OK;
+}
+
+nm_status_t nm_weights_reserve(nm_weights_t* w, size_t bytes)
+{
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_reserve: bad weights handle");
+    if (bytes <= w->splitk_bytes) return NM_OK;
+    cudaDeviceSynchronize();
+    cudaFree(w->splitk);
+    w->splitk = nullptr;
+    w->splitk_bytes = 0;
+    if (cudaMalloc(&w->splitk, bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nmhost::fail(NM_ERR_ALLOC, "nm_weights_reserve: cannot allocate %zu bytes", bytes);
+    }
+    w->splitk_bytes = bytes;
+    return NM_OK;
+}
+
 nm_status_t nm_weights_check(const nm_weights_t* w, void* cuda_stream)
 {
     if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_check: bad weights handle");
@@ -373,14 +403,7 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
         const long long pix_blocks = (p.pixels + 127) / 128;
         const bool few_items = pix_blocks * ((p.c_out + 255) / 256) < n_sm && p.k / 32 >= 32;
         const size_t need = few_items && p.wx ? nmhost::expand_splitk_bytes(p, 4) : 0;
-        if (need > hw->splitk_bytes) {
-            cudaStreamSynchronize(st);
-            cudaFree(hw->splitk);
-            hw->splitk = nullptr;
-            hw->splitk_bytes = 0;
-            if (cudaMalloc(&hw->splitk, need) == cudaSuccess) hw->splitk_bytes = need;
-            else (void)cudaGetLastError();   // no scratch: the split plans are simply not candidates
-        }
+        if (need > hw->splitk_bytes) (void)nm_weights_reserve(hw, need);   // no scratch: the split plans are simply not candidates
         p.splitk = hw->splitk;
         p.splitk_bytes = hw->splitk_bytes;
     }

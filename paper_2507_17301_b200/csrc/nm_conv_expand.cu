@@ -345,7 +345,8 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
 {
     ExpandCfg cfg;
     if (!make_cfg(p, plan, &cfg))
-        return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the expanded-operand kernel does not take this layer / plan");
+        return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the expanded-operand kernel does not take this layer / plan%s",
+                    plan && plan->split > 1 ? " (a split plan needs scratch: nm_weights_reserve)" : "");
     // a split-K plan stores raw partial sums [split][pixel][channel] in the handle's scratch; bias and
     // activation are applied by the reduction pass
     ConvParams q = p;

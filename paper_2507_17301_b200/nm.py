@@ -53,12 +53,16 @@ def _load():
     lib.nm_weights_export.argtypes = [vp, vp, vp, vp]
     lib.nm_weights_import.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, ctypes.POINTER(vp)]
     lib.nm_weights_check.argtypes = [vp, vp]
+    lib.nm_plan_scratch_bytes.argtypes = [vp] + [i] * 9 + [pp, ctypes.POINTER(ctypes.c_size_t)]
+    lib.nm_weights_reserve.argtypes = [vp, ctypes.c_size_t]
     lib.nm_weights_free.argtypes = [vp]
     conv_geom = [i] * 9
     lib.nm_conv2d.argtypes = [vp, vp] + conv_geom + [vp, i, vp, pp, vp]
     lib.nm_conv2d_host.argtypes = [vp, vp, vp] + conv_geom + [vp, vp, i, vp, vp, pp, vp]
     lib.nm_autotune.argtypes = [vp, vp] + conv_geom + [vp, i, vp, vp, pp, fp]
     lib.nm_autotune_tile.argtypes = [vp, i, i, i, i, i, i, ip, i, vp] + conv_geom + [vp, i, vp, vp, ip, pp, fp]
+    for name in ("nm_plan_scratch_bytes", "nm_weights_reserve"):
+        getattr(lib, name).restype = ctypes.c_int
     for name in ("nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
                  "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile"):
         getattr(lib, name).restype = ctypes.c_int
@@ -73,7 +77,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -183,6 +187,21 @@ def nm_weights_import(values: torch.Tensor, indices: torch.Tensor, kh: int, kw: 
     _check(_lib.nm_weights_import(vptr, indices.data_ptr(), values.shape[0], kh, kw, c_in, n_keep, m_group, tile_t,
                                   _stream(), ctypes.byref(out)))
     return Weights(out.value)
+
+
+def nm_plan_scratch_bytes(w: Weights, x_shape, stride, pad, dil, plan: nm_plan_t) -> int:
+    """Scratch bytes `plan` needs on this layer (0 for most plans)."""
+    stride, pad, dil = _pair(stride), _pair(pad), _pair(dil)
+    b, h, wd, _ = x_shape
+    out = ctypes.c_size_t()
+    _check(_lib.nm_plan_scratch_bytes(w.handle, b, h, wd, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1],
+                                      ctypes.byref(plan), ctypes.byref(out)))
+    return int(out.value)
+
+
+def nm_weights_reserve(w: Weights, nbytes: int):
+    """Reserves handle-owned scratch memory (allocates; call outside the timed / captured region)."""
+    _check(_lib.nm_weights_reserve(w.handle, nbytes))
 
 
 def nm_weights_check(w: Weights):

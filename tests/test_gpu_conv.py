@@ -233,7 +233,13 @@ def test_split_k_plans(nm, integer):
     with pytest.raises(nm.NmError) as e:                      # no scratch yet: the plan is refused
         nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
     assert e.value.status == nm.NM_ERR_UNSUPPORTED
-    best, ms = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)   # reserves the scratch
+    need = nm.nm_plan_scratch_bytes(hnd, xd.shape, s.stride, s.pad, s.dil, plan)
+    assert need == 2 * 512 * 64 * 4                           # splits x pixels padded to 128 x channels x 4 bytes
+    nm.nm_weights_reserve(hnd, need)                          # explicit reservation: now the plan runs
+    y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
+    torch.cuda.synchronize()
+    assert_conv_close(y.cpu().numpy(), yr)
+    best, ms = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)   # reserves for 4 splits
     assert ms > 0
     for splits in (2, 3, 4):
         for bn in (32, 64):
