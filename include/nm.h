@@ -71,8 +71,12 @@ typedef struct nm_weights nm_weights_t;
  *            5 = row-run kernel for few input channels (c_in % 32 != 0, dil_w = 1, output rows of
  *                at most 128 pixels, K <= 512, c_out % 32 == 0 and <= 256, w * c_in * 4 a multiple
  *                of 16).
+ *            6 = window kernel for stride-1 convolutions with a spatial kernel (3x3 and the like): one
+ *                input patch per 32-channel block in shared memory, every tap a shifted view of it
+ *                (needs stride 1, c_in % 32 == 0, c_out % 32 == 0, w + 2 * pad_w <= 256; expanded
+ *                weights as in variant 4).
  *   bn       output channels per CTA / work item (variants 2, 3: a multiple of tile_t; variant 4: a
- *            multiple of 32 up to 256), 0 = default
+ *            multiple of 32 up to 256; variant 6 likewise), 0 = default
  *   stages   depth of the shared-memory ring, 0 = default
  *   split    variant 2: 1 = cp.async producer, 2 = direct-store epilogue; variant 4: number of CTAs the
  *            reduction axis is split over (2-8; partial sums go through scratch memory that nm_autotune
@@ -196,7 +200,7 @@ nm_status_t nm_weights_free(nm_weights_t* w);
  * with (kh_j, kw_j, c_j) decoded from indices[o / tile_t][j] and reads outside the image = 0.
  * Arithmetic: operands rounded to TF32 (weights once at prune time, round-to-nearest; activations
  * round-to-nearest where they pass through registers (variants 1-3), truncated where the staged
- * slab feeds the tensor core directly (variants 4, 5)), products accumulated in fp32.
+ * slab feeds the tensor core directly (variants 4, 5, 6)), products accumulated in fp32.
  *
  *   x      device fp32 [batch][h][wd][c_in]      bias  device fp32 [c_out] or NULL
  *   y      device fp32 [batch][ho][wo][c_out]    relu  0 = identity, 1 = ReLU
