@@ -81,7 +81,7 @@ typedef struct nm_weights nm_weights_t;
  *   split    variant 2: 1 = cp.async producer, 2 = direct-store epilogue; variant 4: number of CTAs the
  *            reduction axis is split over (2-8; partial sums go through scratch memory that nm_autotune
  *            reserves on the handle, so such a plan works only on a handle nm_autotune has seen with a
- *            layer at least as large); variant 6: M-tiles per work item (1 or 2); otherwise 0
+ *            layer at least as large); variant 6: M-tiles per work item (1-4); otherwise 0
  * A plan the layer does not admit gives NM_ERR_UNSUPPORTED.
  */
 typedef struct {

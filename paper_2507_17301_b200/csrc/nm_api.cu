@@ -158,7 +158,7 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     std::vector<nm_plan_t> out;
     nm_plan_t a;
     std::memset(&a, 0, sizeof(a));
-    for (int mt : {1, 2}) {                 // window kernel (stride-1 spatial kernels)
+    for (int mt : {2, 3, 4, 1}) {           // window kernel (stride-1 spatial kernels)
         for (int bn : {64, 128, 256}) {
             a.variant = 6; a.bn = bn; a.split = mt; a.stages = 0;
             if (nmhost::window_plan_ok(p, &a)) out.push_back(a);

@@ -240,7 +240,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
             }
         }
-        if (lane == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads; the writes complete with the grid
     }
 
     tc_fence_before();

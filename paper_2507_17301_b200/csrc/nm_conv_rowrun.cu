@@ -248,7 +248,7 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                 }
             }
         }
-        if (lane == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads; the writes complete with the grid
     } else if (warp >= 8) {
         // =========================== builders ===========================
         // Two groups of eight warps build alternate sub-tiles, so that one group's barrier waits and

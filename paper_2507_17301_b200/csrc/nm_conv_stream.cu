@@ -318,7 +318,7 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                 }
             }
         }
-        if (lane == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads; the writes complete with the grid
     } else if (warp >= 8) {
         // =========================== compactors ===========================
         const int wg = (warp - 8) >> 2;   // which half of the chunk

@@ -15,10 +15,12 @@
 //                               expanded, pre-swizzled weights [BN x 32] (zeros = pruned columns)
 //   MMA issuers (1 thread per   per block and tap four 128 x BN x 8 TF32 tcgen05.mma
 //   M-tile)
-//   epilogue (4 warps)          TMEM -> registers, + bias, ReLU, staging in output-row order, one TMA
-//                               store per output row and 32-channel block
+//   epilogue (4 warps)          TMEM -> registers, + bias, ReLU, 16-byte stores straight to NHWC (each
+//                               thread owns one position = 128 contiguous bytes per 32-channel block;
+//                               no staging buffer, so shared memory goes to patches and weights)
 // A work item is (image, block of R output rows, BN channels) with R * Wp <= 128 * MT positions
-// (MT = 1 or 2 M-tiles sharing patch and weights).  Persistent CTAs, static schedule, bounded waits.
+// (MT = 1..4 M-tiles sharing patch and weights, each with its own issuer thread and accumulator).
+// Persistent CTAs, static schedule, bounded waits.
 #include "nm_internal.h"
 #include "nm_ptx.cuh"
 #include "nm_tmap.cuh"
@@ -28,23 +30,23 @@ namespace {
 using namespace nmk;
 
 constexpr int BM = 128;
-constexpr int THREADS = 256;
+constexpr int MAX_MT = 4;
+constexpr int THREADS = 384;   // warps: 0 patch producer, 1 weight producer, 2-5 MMA issuers, 6 TMEM, 8-11 epilogue
 constexpr int MAX_P = 4;    // patch ring slots
 constexpr int MAX_W = 12;   // weight ring slots
 
 struct WinCfg {
     int bn, n_slices;
-    int mt;            // M-tiles per item (1 or 2)
+    int mt;            // M-tiles per item (1 .. 4)
+    int n_acc;         // accumulator sets in tensor memory: 2 when 2 * mt * bn <= 512, else 1
     int r_rows;        // output rows per item
     int wp;            // padded width = positions per output row
-    int wp8;           // staging rows per output row (wp rounded up to 8)
     int pr;            // patch rows = r_rows + (kh - 1) * dil_h
     int patch_bytes;   // TMA box bytes = pr * wp * 128
     int pslot_bytes;   // patch slot incl. overrun rows, multiple of 1024
     int n_p, n_w;      // ring depths
     int n_kb;          // c_in / 32
     int row_blocks;    // ceil(ho / r_rows)
-    int stage_bytes;   // one staging buffer = r_rows * wp8 * 128
     long long n_work;
 };
 
@@ -57,30 +59,6 @@ __device__ __forceinline__ void tma_load_tiled_4d(uint32_t dst, const void* tmap
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n)
         : "memory");
 }
-__device__ __forceinline__ void tma_store_4d(const void* tmap, uint32_t src, int c, int w, int h, int n)
-{
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tmap),
-                 "r"(src), "r"(c), "r"(w), "r"(h), "r"(n)
-                 : "memory");
-}
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// Barrier of the 128 epilogue threads that also ORs a flag, so that all of them take the same exit.
-__device__ __forceinline__ bool epi_bar_or(bool flag)
-{
-    uint32_t out;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred pin, pout;\n\t"
-        "setp.ne.u32 pin, %1, 0;\n\t"
-        "bar.red.or.pred pout, 1, 128, pin;\n\t"
-        "selp.u32 %0, 1, 0, pout;\n\t"
-        "}\n"
-        : "=r"(out)
-        : "r"(flag ? 1u : 0u)
-        : "memory");
-    return out != 0;
-}
-
 // K-major, 128-byte-swizzled operand whose first row may sit on any 128-byte boundary of a
 // 1024-byte-aligned buffer: the tensor core derives the swizzle phase of a row from its
 // shared-memory address (as the TMA unit did when it wrote the row), so a view shifted by whole
@@ -102,8 +80,7 @@ __device__ __forceinline__ ItemPos item_of(uint32_t work, const WinCfg& cfg)
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUtensorMap tm_x,
-              const __grid_constant__ CUtensorMap tm_y)
+k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUtensorMap tm_x)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_pfull[MAX_P], s_pfree[MAX_P], s_wfull[MAX_W], s_wfree[MAX_W], s_accfull[2], s_accfree[2];
@@ -117,12 +94,11 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
     const uint32_t w_ring = p_ring + cfg.n_p * cfg.pslot_bytes;
     const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
     const uint32_t wslot_bytes = (w_bytes + 1023u) & ~1023u;
-    const uint32_t staging = w_ring + cfg.n_w * wslot_bytes;
     const int n_taps = p.kh * p.kw;
     const int acc_cols = cfg.mt * cfg.bn;
     volatile int* abort_flag = &s_abort;
 
-    if (warp == 2) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (warp == 6) tmem_alloc(smem_u32(&s_tmem), 512);
     if (tid == 0) {
         for (int i = 0; i < MAX_P; ++i) { mbar_init(smem_u32(&s_pfull[i]), 1); mbar_init(smem_u32(&s_pfree[i]), cfg.mt); }
         for (int i = 0; i < MAX_W; ++i) { mbar_init(smem_u32(&s_wfull[i]), 1); mbar_init(smem_u32(&s_wfree[i]), cfg.mt); }
@@ -130,7 +106,6 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
         mbar_fence_init();
         s_abort = 0;
         tma_prefetch_desc(&tm_x);
-        tma_prefetch_desc(&tm_y);
     }
     tc_fence_before();
     __syncthreads();
@@ -164,7 +139,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp == 3) {
+    } else if (warp == 1) {
         // =========================== weight producer ===========================
         if (lane == 0) {
             RingPos rw;
@@ -195,13 +170,13 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp == 1 || (warp == 2 && cfg.mt == 2)) {
+    } else if (warp >= 2 && warp < 2 + cfg.mt) {
         // =========================== MMA issuers ===========================
         // One thread per M-tile: a single thread cannot issue small MMAs as fast as the tensor core
         // retires them, and the M-tiles have separate accumulators, so each gets its own issuer.
         // Ring slots and accumulator hand-offs count one commit per issuer.
         if (lane == 0) {
-            const int mi = warp - 1;
+            const int mi = warp - 2;
             const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
             // one tap to the right = dil_w patch rows of 128 bytes; after the last tap of a kernel row,
             // back to the first column and dil_h patch lines (Wp rows each) down
@@ -241,73 +216,64 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
                 }
                 if (aborted(abort_flag)) break;
                 umma_commit(smem_u32(&s_accfull[ab]));
-                if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
-                ab ^= 1u;
+                if (cfg.n_acc == 2) {
+                    if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
+                    ab ^= 1u;
+                } else {
+                    acc_par ^= 1u;
+                    acc_wrapped = true;
+                }
             }
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 8) {
         // =========================== epilogue ===========================
         const int q = warp & 3;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const int n_blk = cfg.bn / 32;
-        uint32_t ti = 0, nb = 0;   // items done, staging buffers filled
+        uint32_t ti = 0;
         for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
             const ItemPos it = item_of(work, cfg);
-            const int ab = static_cast<int>(ti & 1u);
-            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
-            if (!ok) *abort_flag = 8;
-            if (epi_bar_or(!ok || aborted(abort_flag))) break;   // all four warps leave together or not at all
+            const int ab = cfg.n_acc == 2 ? static_cast<int>(ti & 1u) : 0;
+            const bool ok = aborted(abort_flag) ||
+                            mbar_wait(smem_u32(&s_accfull[ab]), (cfg.n_acc == 2 ? (ti >> 1) : ti) & 1u);
+            if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
+            if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
             const int o0 = it.slice * cfg.bn;
-            for (int blk = 0; blk < n_blk; ++blk, ++nb) {
-                const uint32_t buf = staging + (nb & 1u) * cfg.stage_bytes;
-                if (tid == 128 && nb >= 2) tma_store_wait_read_n<1>();   // the stores that last read this buffer are done
-                epi_bar();
-                for (int m = 0; m < cfg.mt; ++m) {
+            for (int m = 0; m < cfg.mt; ++m) {
+                // this thread's position: row of the block and column along the padded width
+                const int pos = m * BM + q * 32 + lane;
+                const int r = pos / cfg.wp, ow = pos - r * cfg.wp;
+                const bool valid = r < cfg.r_rows && ow < p.wo && it.oh0 + r < p.ho;
+                float* yrow = p.y + ((static_cast<size_t>(it.n) * p.ho + (valid ? it.oh0 + r : 0)) * p.wo + (valid ? ow : 0)) * p.c_out + o0;
+                for (int blk = 0; blk < n_blk; ++blk) {
                     uint32_t v[32];
                     tmem_ld32(tmem + lane_addr + ab * acc_cols + m * cfg.bn + blk * 32, v);
                     tmem_ld_wait();
-                    if (blk == n_blk - 1 && m == cfg.mt - 1) {
+                    if (m == cfg.mt - 1 && blk == n_blk - 1) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
                     }
-                    const int pos = m * BM + q * 32 + lane;
-                    const int r = pos / cfg.wp, ow = pos - r * cfg.wp;
-                    if (r < cfg.r_rows) {
-                        const int srow = r * cfg.wp8 + ow;
-                        const uint32_t row_addr = buf + static_cast<uint32_t>(srow) * 128u;
-                        const uint32_t rx = static_cast<uint32_t>(srow & 7);
+                    if (valid) {
 #pragma unroll
                         for (int qq = 0; qq < 8; ++qq) {
-                            float o[4];
+                            float4 o;
                             float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                             if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
-                            o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
-                            o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
-                            o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
-                            o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
+                            o.x = __uint_as_float(v[qq * 4 + 0]) + bv.x;
+                            o.y = __uint_as_float(v[qq * 4 + 1]) + bv.y;
+                            o.z = __uint_as_float(v[qq * 4 + 2]) + bv.z;
+                            o.w = __uint_as_float(v[qq * 4 + 3]) + bv.w;
                             if (p.relu) {
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
+                                o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
                             }
-                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((qq ^ rx) << 4)),
-                                         "f"(o[0]), "f"(o[1]), "f"(o[2]), "f"(o[3])
-                                         : "memory");
+                            *reinterpret_cast<float4*>(yrow + blk * 32 + qq * 4) = o;
                         }
                     }
                 }
-                fence_proxy_async();
-                epi_bar();
-                if (tid == 128) {
-                    for (int r = 0; r < cfg.r_rows; ++r)
-                        if (it.oh0 + r < p.ho)
-                            tma_store_4d(&tm_y, buf + static_cast<uint32_t>(r * cfg.wp8) * 128u, o0 + blk * 32, 0, it.oh0 + r, it.n);
-                    tma_store_commit();
-                }
             }
         }
-        if (tid == 128) tma_store_wait_all();
     }
 
     tc_fence_before();
@@ -317,7 +283,7 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
         atomicExch(p.status + 1, 60 + s_abort);
         atomicExch(p.status + 2, static_cast<int>(blockIdx.x));
     }
-    if (warp == 2) tmem_dealloc(tmem, 512);
+    if (warp == 6) tmem_dealloc(tmem, 512);
 }
 
 int sm_count()
@@ -342,8 +308,9 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, WinCfg* cfg, size_t* s
     if (p.pad_w > 127 || p.pad_h > 127) return false;
     const int wp = p.w + 2 * p.pad_w;
     if (wp - p.dil_w * (p.kw - 1) != p.wo || p.wo > 256) return false;
-    int mt = plan && plan->split > 0 ? plan->split : (wp > BM ? 2 : 1);
-    if (mt < 1 || mt > 2 || wp > BM * mt) return false;
+    int mt = plan && plan->split > 0 ? plan->split : 2;
+    if (mt * BM < wp) mt = (wp + BM - 1) / BM;          // one output row must fit the item
+    if (mt < 1 || mt > MAX_MT) return false;
     int r_rows = (BM * mt) / wp;
     if (r_rows > p.ho) r_rows = p.ho;
     const int pr = r_rows + (p.kh - 1) * p.dil_h;
@@ -353,15 +320,15 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, WinCfg* cfg, size_t* s
         bn = plan->bn;
     } else {
         for (int cand : {256, 128, 64, 32, 96, 160, 192, 224})
-            if (cand <= p.c_out && p.c_out % cand == 0 && 2 * mt * cand <= 512) { bn = cand; break; }
+            if (cand <= p.c_out && p.c_out % cand == 0 && mt * cand <= 512) { bn = cand; break; }
     }
-    if (bn < 32 || bn > 256 || bn % 32 != 0 || p.c_out % bn != 0 || 2 * mt * bn > 512) return false;
+    if (bn < 32 || bn > 256 || bn % 32 != 0 || p.c_out % bn != 0 || mt * bn > 512) return false;
+    cfg->n_acc = 2 * mt * bn <= 512 ? 2 : 1;
     cfg->bn = bn;
     cfg->n_slices = p.c_out / bn;
     cfg->mt = mt;
     cfg->r_rows = r_rows;
     cfg->wp = wp;
-    cfg->wp8 = (wp + 7) / 8 * 8;
     cfg->pr = pr;
     cfg->patch_bytes = pr * wp * 128;
     if (cfg->patch_bytes >= (1 << 20)) return false;
@@ -371,11 +338,10 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, WinCfg* cfg, size_t* s
     cfg->pslot_bytes = ((rows * 128 + 1023) / 1024) * 1024;
     cfg->n_kb = p.c_in / 32;
     cfg->row_blocks = (p.ho + r_rows - 1) / r_rows;
-    cfg->stage_bytes = r_rows * cfg->wp8 * 128;
     cfg->n_work = static_cast<long long>(p.batch) * cfg->row_blocks * cfg->n_slices;
     if (cfg->n_work >= (1ll << 31)) return false;
     const int wslot = ((bn * 128 + 1023) / 1024) * 1024;
-    const int budget = 227 * 1024 - 2048 - 2 * cfg->stage_bytes;
+    const int budget = 227 * 1024 - 2048;
     int n_p = 2, n_w = plan && plan->stages > 0 ? plan->stages : MAX_W;
     if (n_w > MAX_W || n_w < 2) return false;
     while (n_w > 3 && n_p * cfg->pslot_bytes + n_w * wslot > budget) --n_w;
@@ -383,7 +349,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, WinCfg* cfg, size_t* s
     while (n_p < MAX_P && (n_p + 1) * cfg->pslot_bytes + n_w * wslot <= budget) ++n_p;
     cfg->n_p = n_p;
     cfg->n_w = n_w;
-    size_t smem = 1024 + static_cast<size_t>(n_p) * cfg->pslot_bytes + static_cast<size_t>(n_w) * wslot + 2 * cfg->stage_bytes;
+    size_t smem = 1024 + static_cast<size_t>(n_p) * cfg->pslot_bytes + static_cast<size_t>(n_w) * wslot;
     *smem_out = smem < 120 * 1024 ? 120 * 1024 : smem;
     return true;
 }
@@ -403,20 +369,6 @@ bool encode_x_patch(const ConvParams& p, const WinCfg& cfg, CUtensorMap* tm)
                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Output as (C_out, Wo, Ho, N) with a 32-channel x Wo x 1 x 1 box: one output row per store.
-bool encode_y_row(const ConvParams& p, CUtensorMap* tm)
-{
-    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.c_out), static_cast<cuuint64_t>(p.wo),
-                                static_cast<cuuint64_t>(p.ho), static_cast<cuuint64_t>(p.batch)};
-    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(p.c_out) * 4, static_cast<cuuint64_t>(p.wo) * p.c_out * 4,
-                                   static_cast<cuuint64_t>(p.ho) * p.wo * p.c_out * 4};
-    const cuuint32_t box[4] = {32, static_cast<cuuint32_t>(p.wo), 1, 1};
-    const cuuint32_t es[4] = {1, 1, 1, 1};
-    return nmtm::encoders().tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.y, dims, strides, box, es,
-                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 namespace nmhost {
@@ -434,13 +386,13 @@ nm_status_t launch_conv_window(const ConvParams& p, const nm_plan_t* plan, cudaS
     size_t smem = 0;
     if (!make_cfg(p, plan, &cfg, &smem))
         return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the window kernel does not take this layer / plan");
-    alignas(64) CUtensorMap tm_x, tm_y;
-    if (!encode_x_patch(p, cfg, &tm_x) || !encode_y_row(p, &tm_y))
+    alignas(64) CUtensorMap tm_x;
+    if (!encode_x_patch(p, cfg, &tm_x))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 6)");
     cudaError_t e = cudaFuncSetAttribute(k_conv_window, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 6): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    e = launch_pdl(k_conv_window, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x, tm_y);
+    e = launch_pdl(k_conv_window, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x);
     count_launch(1);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 6): %s", cudaGetErrorString(e));

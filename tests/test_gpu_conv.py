@@ -37,8 +37,8 @@ def _plans(nm, s):
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
     out.append(p)
-    # window kernel: default, one M-tile with 64 channels, two M-tiles, short weight ring
-    for bn, mt, stages in ((0, 0, 0), (64, 1, 0), (0, 2, 0), (32, 1, 3)):
+    # window kernel: default, one M-tile with 64 channels, two / three / four M-tiles, short weight ring
+    for bn, mt, stages in ((0, 0, 0), (64, 1, 0), (0, 2, 0), (32, 1, 3), (64, 3, 0), (32, 4, 0), (128, 4, 0)):
         p = nm.nm_plan_t()
         p.variant, p.bn, p.split, p.stages = 6, bn, mt, stages
         out.append(p)
