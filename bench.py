@@ -303,6 +303,7 @@ def main():
     ap.add_argument("--depth", type=int, default=50, choices=[50, 101, 152], help="ResNet depth of the conv stack")
     ap.add_argument("--nm", default="2:4", help="N:M pattern of the pruned layers, e.g. 1:4 or 2:8")
     ap.add_argument("--tile", type=int, default=64, help="pruning tile width T")
+    ap.add_argument("--json-out", default=None, help="also write the result, indented, to this file")
     ap.add_argument("--save-plans", default=None, help="write the auto-tuned plans to this JSON file")
     ap.add_argument("--load-plans", default=None, help="use the plans of this JSON file instead of auto-tuning")
     args = ap.parse_args()
@@ -551,9 +552,9 @@ def main():
         out["cpu_baseline"] = cpu_baseline()
 
     if rank == 0:
-        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-        with open(os.path.join(ROOT, "gpurun_out", "bench_last.json"), "w") as f:
-            json.dump(out, f, indent=1)
+        if args.json_out:
+            with open(args.json_out, "w") as f:
+                json.dump(out, f, indent=1)
         print(json.dumps(out))
     if world > 1:
         import torch.distributed as dist

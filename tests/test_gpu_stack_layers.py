@@ -1,0 +1,57 @@
+"""Layers of the benchmark workload at the benchmark's own size (ResNet-50 shapes, batch 64) and in its
+launch configuration (the plan nm_autotune picks), checked on sampled outputs: whole images of the
+batch that the CPU oracle computes one by one."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2507_17301_b200 import inputs
+from parity import assert_conv_close, assert_prune_bit_exact
+
+pytestmark = pytest.mark.gpu
+
+# stem (dense, few channels), 1x1 wide output, 3x3 at 56x56, strided 3x3, strided 1x1 projection,
+# tensor-bound 3x3 at 14x14, long-reduction 1x1 and 3x3 at 7x7 (split-K candidates)
+LAYERS = ["stem7x7", "s1b1_c3", "s1b1_c2", "s2b1_c2", "s2b1_ds", "s3b2_c2", "s4b2_c1", "s4b2_c2"]
+IMAGES = (0, 37, 63)
+
+
+@pytest.fixture(scope="module")
+def nm():
+    from paper_2507_17301_b200 import nm as mod
+    return mod
+
+
+@pytest.fixture(scope="module")
+def stack():
+    layers = inputs.resnet_conv_stack(50, 64, 2, 4, tile_t=64)
+    return {s.name: (i, s) for i, s in enumerate(layers)}
+
+
+@pytest.mark.parametrize("name", LAYERS)
+def test_stack_layer_sampled_images(nm, stack, name):
+    li, s = stack[name]
+    w = inputs.make_weights(s, li)
+    b = inputs.make_bias(s, li)
+    g = torch.Generator().manual_seed(1 + 1000 * li)
+    x = torch.randn((s.batch, s.h, s.w, s.c_in), generator=g)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    v, i = nm.nm_weights_export(hnd)
+    vr, ir = oracle.prune(w.numpy(), s.n_keep, s.m_group, s.tile_t)
+    assert_prune_bit_exact(v.cpu().numpy(), i.cpu().numpy(), vr, ir)
+    xd, bd = x.cuda(), b.cuda()
+    plan, ms = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)
+    assert ms > 0
+    y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
+    nm.nm_weights_check(hnd)
+    torch.cuda.synchronize()
+    for n in IMAGES:
+        yr = oracle.conv2d(vr, ir, s.kh, s.kw, s.c_in, s.tile_t, x[n:n + 1].numpy(), (s.stride,) * 2, (s.pad,) * 2,
+                           (s.dil,) * 2, b.numpy(), s.relu)
+        assert_conv_close(y[n:n + 1].cpu().numpy(), yr)
+    # the rest of the batch: finite everywhere, and no image left unwritten (a ReLU layer may hold zeros,
+    # an all-zero image would mean a skipped work item)
+    yc = y.cpu()
+    assert torch.isfinite(yc).all()
+    assert (yc.abs().amax(dim=(1, 2, 3)) > 0).all()
