@@ -78,8 +78,9 @@ typedef struct nm_weights nm_weights_t;
  *   bn       output channels per CTA / work item (variants 2, 3: a multiple of tile_t; variant 4: a
  *            multiple of 32 up to 256; variant 6 likewise), 0 = default
  *   stages   depth of the shared-memory ring, 0 = default
- *   split    variant 2: 1 = cp.async producer, 2 = direct-store epilogue; variant 4: number of CTAs the
- *            reduction axis is split over (2-8; partial sums go through scratch memory that nm_autotune
+ *   split    variant 2: 1 = cp.async producer, 2 = direct-store epilogue; variant 4: 0 = keep a CTA's weight
+ *            slice resident in shared memory when it fits, 1 = stream the weights with the activations,
+ *            2-8 = number of CTAs the reduction axis is split over ( partial sums go through scratch memory that nm_autotune
  *            reserves on the handle, so such a plan works only on a handle nm_autotune has seen with a
  *            layer at least as large); variant 6: M-tiles per work item (1-4); otherwise 0
  * A plan the layer does not admit gives NM_ERR_UNSUPPORTED.

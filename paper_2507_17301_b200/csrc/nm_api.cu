@@ -168,9 +168,11 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     a.variant = 5;                          // row-run kernel (few input channels)
     if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, &a)) out.push_back(a);
     std::memset(&a, 0, sizeof(a));
-    for (int bn : {64, 128, 256}) {         // expanded-operand kernel
-        a.variant = 4; a.bn = bn; a.stages = 0; a.split = 0;
-        if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);
+    for (int split : {0, 1}) {              // expanded-operand kernel: weights resident where they fit / streamed
+        for (int bn : {64, 128, 256}) {
+            a.variant = 4; a.bn = bn; a.stages = 0; a.split = split;
+            if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);
+        }
     }
     for (int splits : {2, 3, 4}) {          // ... with the reduction axis split (needs the handle's scratch)
         for (int bn : {128, 256}) {

@@ -13,7 +13,9 @@
 // The pruning tile width plays no role here, so any tile_t is accepted.
 //
 //   producer (1 thread)   TMA im2col load of the slab + one contiguous bulk copy of the weight block
-//                         (stored pre-swizzled, so it costs no per-row TMA requests) per stage
+//                         (stored pre-swizzled, so it costs no per-row TMA requests) per stage; a
+//                         weight slice of at most 128 KB is instead fetched once and stays resident
+//                         (the grid is then a multiple of the slice count, so a CTA keeps its slice)
 //   MMA issuer (1 thread) four 128 x BN x 8 TF32 tcgen05.mma (SS) per stage into one of two
 //                         accumulator buffers in tensor memory
 //   epilogue (8 warps)    TMEM -> registers, + bias, ReLU, swizzled staging, TMA store to NHWC;
@@ -30,7 +32,8 @@ using namespace nmk;
 
 constexpr int BM = 128;
 constexpr int SUB_BYTES = BM * 128;
-constexpr int NSTAGE_MAX = 8;
+constexpr int NSTAGE_MAX = 10;
+constexpr int WRES_MAX = 128 * 1024;            // largest weight slice kept resident
 constexpr int THREADS = 384;                   // 4 service warps + 8 epilogue warps
 constexpr int BOX_BYTES = 4096;                // one 32-pixel x 32-channel output box
 
@@ -40,6 +43,8 @@ struct ExpandCfg {
     int stages;
     int b_bytes;      // weight bytes per stage (bn rows of 128 bytes)
     int stage_bytes;
+    int w_res;        // 1: this CTA's weight slice stays resident in shared memory (it is loaded once)
+    int wres_bytes;   // bytes of the resident slice: all 32-column blocks of bn rows
     int n_sub;        // 32-column blocks one work item reduces over: (K / 32) / ksplit
     int ksplit;       // K splits (1 = none): a work item covers one of them and stores raw partial sums
     int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
@@ -54,14 +59,15 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
               const __grid_constant__ CUtensorMap tm_y)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t s_full[NSTAGE_MAX], s_free[NSTAGE_MAX], s_accfull[2], s_accfree[2];
+    __shared__ uint64_t s_full[NSTAGE_MAX], s_free[NSTAGE_MAX], s_accfull[2], s_accfree[2], s_wres;
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t n_work = static_cast<uint32_t>(cfg.n_work);   // below 2^31: per-item arithmetic stays 32-bit
     const int NS = cfg.stages, n_sub = cfg.n_sub;
-    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t wres = (smem_u32(smem_raw) + 1023u) & ~1023u;   // resident weight slice (may be empty)
+    const uint32_t ring = wres + cfg.wres_bytes;
     const uint32_t staging = ring + NS * cfg.stage_bytes;
     volatile int* abort_flag = &s_abort;
 
@@ -75,6 +81,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             mbar_init(smem_u32(&s_accfull[i]), 1);   // MMA commit
             mbar_init(smem_u32(&s_accfree[i]), 8);   // epilogue warps
         }
+        mbar_init(smem_u32(&s_wres), 1);
         mbar_fence_init();
         s_abort = 0;
         tma_prefetch_desc(&tm_x);
@@ -92,7 +99,16 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         if (lane == 0) {
             int issued = 0;
             const int hw = p.ho * p.wo;
-            const uint32_t tx = SUB_BYTES + static_cast<uint32_t>(cfg.bn) * 128u;
+            const uint32_t tx = SUB_BYTES + (cfg.w_res ? 0u : static_cast<uint32_t>(cfg.bn) * 128u);
+            if (cfg.w_res) {
+                // the grid is a multiple of the slice count, so every work item of this CTA has the
+                // same channel slice: its weights are fetched once
+                const int slice = static_cast<int>(blockIdx.x % static_cast<uint32_t>(cfg.n_slices));
+                mbar_arrive_expect_tx(smem_u32(&s_wres), static_cast<uint32_t>(n_sub) * static_cast<uint32_t>(cfg.bn) * 128u);
+                for (int c = 0; c < n_sub; ++c)
+                    bulk_load_1d(wres + c * cfg.b_bytes, p.wx + (static_cast<size_t>(c) * p.c_out + slice * cfg.bn) * 32,
+                                 static_cast<uint32_t>(cfg.bn) * 128u, smem_u32(&s_wres));
+            }
             const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
             const size_t w_step = static_cast<size_t>(p.c_out) * 32;   // floats between two 32-column blocks
             RingPos rp;
@@ -119,7 +135,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     mbar_arrive_expect_tx(bar, tx);
                     tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>(off_w),
                                        static_cast<uint16_t>(off_h));
-                    bulk_load_1d(a_smem + SUB_BYTES, wsrc, w_bytes, bar);
+                    if (!cfg.w_res) bulk_load_1d(a_smem + SUB_BYTES, wsrc, w_bytes, bar);
                     wsrc += w_step;
                     ch += 32;
                     if (ch >= p.c_in) {
@@ -133,6 +149,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             }
             if (aborted(abort_flag)) {
                 // loads already issued still target this CTA's shared memory: let them land
+                if (cfg.w_res) (void)mbar_wait(smem_u32(&s_wres), 0);
                 for (int back = 0; back < NS && back < issued; ++back) {
                     if (rp.s == 0) { rp.s = NS; rp.parity ^= 1u; }
                     --rp.s;
@@ -144,6 +161,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
+            if (cfg.w_res && !mbar_wait(smem_u32(&s_wres), 0)) *abort_flag = 9;
             RingPos rp;
             uint32_t ab = 0, acc_par = 0;   // accumulator buffer of this item, parity of its current use
             bool acc_wrapped = false;
@@ -159,7 +177,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     tc_fence_after();
                     const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     const uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
-                    const uint64_t bdesc = umma_desc_k_sw128(a_smem + SUB_BYTES, 1024);
+                    const uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
 #pragma unroll
                     for (int kq = 0; kq < 4; ++kq)
                         umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > 0 || kq > 0) ? 1u : 0u);
@@ -306,7 +324,6 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     cfg->bn = bn;
     cfg->n_slices = p.c_out / bn;
     cfg->b_bytes = ((bn * 128 + 1023) / 1024) * 1024;
-    cfg->stage_bytes = SUB_BYTES + cfg->b_bytes;
     const int splits = plan && plan->split > 1 ? plan->split : 1;
     if (splits > 8 || (p.k / 32) % splits != 0) return false;
     cfg->ksplit = splits;
@@ -316,7 +333,18 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
                        static_cast<long long>(splits) * cfg->p_pad >= (1ll << 31)))
         return false;   // the partial-sum scratch is reserved by nm_autotune
     cfg->boxes = cfg->n_sub <= 8 ? 2 : 1;   // long reductions: the epilogue is rare, the ring needs the bytes
-    const int budget = 227 * 1024 - 1024 - 8 * cfg->boxes * BOX_BYTES - 1024;
+    // A weight slice that fits stays resident (plan.split == 1 asks for streaming instead): the ring
+    // then holds activations only and is deeper.  Needs one fixed slice per CTA, i.e. a grid that is a
+    // multiple of the slice count.
+    cfg->wres_bytes = 0;
+    cfg->w_res = 0;
+    if (splits == 1 && !(plan && plan->split == 1) && cfg->n_sub * cfg->b_bytes <= WRES_MAX && cfg->n_slices <= sm_count()) {
+        cfg->w_res = 1;
+        cfg->wres_bytes = cfg->n_sub * cfg->b_bytes;
+        if (cfg->wres_bytes > 64 * 1024) cfg->boxes = 1;   // a large slice: give the output staging's room to the ring
+    }
+    cfg->stage_bytes = SUB_BYTES + (cfg->w_res ? 0 : cfg->b_bytes);
+    const int budget = 227 * 1024 - 1024 - 8 * cfg->boxes * BOX_BYTES - 1024 - cfg->wres_bytes;
     int stages = plan && plan->stages > 0 ? plan->stages : NSTAGE_MAX;
     if (stages > NSTAGE_MAX) return false;
     if (plan && plan->stages > 0) {
@@ -360,11 +388,12 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_y_tiled(q, &tm_y))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 4)");
     q.pixels = p.pixels;
-    size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 8 * cfg.boxes * BOX_BYTES;
+    size_t smem = 1024 + cfg.wres_bytes + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 8 * cfg.boxes * BOX_BYTES;
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
     cudaError_t e = cudaFuncSetAttribute(k_conv_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
-    const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
+    long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
+    if (cfg.w_res) grid = (grid / cfg.n_slices) * cfg.n_slices;   // n_work is a multiple of n_slices, so grid >= n_slices
     e = nmhost::launch_pdl(k_conv_expand, static_cast<unsigned>(grid), THREADS, smem, st, q, cfg, tm_x, tm_y);
     nmhost::count_launch(1);
     if (e == cudaSuccess) e = cudaGetLastError();

@@ -29,10 +29,11 @@ def _plans(nm, s):
         p = nm.nm_plan_t()
         p.variant, p.bn, p.stages = 3, bn, stages
         out.append(p)
-    # expanded-operand kernel: default width, 32 and 256 channels per work item, two-stage ring
-    for bn, stages in ((0, 0), (32, 0), (256, 0), (0, 2)):
+    # expanded-operand kernel: default width, 32 and 256 channels per work item, two-stage ring, and
+    # (split = 1) weights streamed per stage instead of kept resident
+    for bn, stages, split in ((0, 0, 0), (32, 0, 0), (256, 0, 0), (0, 2, 0), (0, 0, 1), (64, 0, 1)):
         p = nm.nm_plan_t()
-        p.variant, p.bn, p.stages = 4, bn, stages
+        p.variant, p.bn, p.stages, p.split = 4, bn, stages, split
         out.append(p)
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
