@@ -102,11 +102,18 @@ WORKLOAD = {"depth": 50, "n": 2, "m": 4, "tile": 64}   # the headline configurat
 
 
 def workload(batch: int):
-    return inputs.resnet_conv_stack(WORKLOAD["depth"], batch, WORKLOAD["n"], WORKLOAD["m"], tile_t=WORKLOAD["tile"])
+    layers = inputs.resnet_conv_stack(WORKLOAD["depth"], batch, WORKLOAD["n"], WORKLOAD["m"], tile_t=WORKLOAD["tile"])
+    r = WORKLOAD.get("adaptive")
+    if r is not None:
+        # the paper's adaptive setting (Sec. 3.1): a group spans a layer's input channels, N = (1 - sparsity) * M
+        layers = [s if s.n_keep == s.m_group else s.with_(m_group=s.c_in, n_keep=max(1, round(s.c_in * (1.0 - r))))
+                  for s in layers]
+    return layers
 
 
 def workload_name(batch: int) -> str:
-    return f"resnet{WORKLOAD['depth']}_conv_stack_b{batch}_224_{WORKLOAD['n']}of{WORKLOAD['m']}"
+    pat = f"{WORKLOAD['n']}of{WORKLOAD['m']}" if WORKLOAD.get("adaptive") is None else f"adaptiveM_sparsity{WORKLOAD['adaptive']}"
+    return f"resnet{WORKLOAD['depth']}_conv_stack_b{batch}_224_{pat}"
 
 
 class ClockSampler:
@@ -303,11 +310,14 @@ def main():
     ap.add_argument("--depth", type=int, default=50, choices=[50, 101, 152], help="ResNet depth of the conv stack")
     ap.add_argument("--nm", default="2:4", help="N:M pattern of the pruned layers, e.g. 1:4 or 2:8")
     ap.add_argument("--tile", type=int, default=64, help="pruning tile width T")
+    ap.add_argument("--adaptive", type=float, default=None,
+                    help="sparsity in (0, 1): groups span a layer's input channels (M = C_in, N = (1 - sparsity) * M)")
     ap.add_argument("--json-out", default=None, help="also write the result, indented, to this file")
     ap.add_argument("--save-plans", default=None, help="write the auto-tuned plans to this JSON file")
     ap.add_argument("--load-plans", default=None, help="use the plans of this JSON file instead of auto-tuning")
     args = ap.parse_args()
-    WORKLOAD.update(depth=args.depth, n=int(args.nm.split(":")[0]), m=int(args.nm.split(":")[1]), tile=args.tile)
+    WORKLOAD.update(depth=args.depth, n=int(args.nm.split(":")[0]), m=int(args.nm.split(":")[1]), tile=args.tile,
+                    adaptive=args.adaptive)
     if args.impl == "reference":
         return run_reference(args)
     if args.warmup < 3:

@@ -260,6 +260,27 @@ def test_split_k_plans(nm, integer):
         assert_conv_close(y.cpu().numpy(), yr)
 
 
+# Groups as wide as the input-channel axis (the paper's adaptive setting, Sec. 3.1: M may span all input
+# channels, N = (1 - sparsity) * M): every kernel that reads the tap table or the expanded weights takes them.
+LARGE_M = [
+    ConvShape("m_is_cin_1x1", 2, 14, 14, 256, 128, 1, 1, 1, 0, 1, 64, 256, 32),       # 75 % sparsity, M = C_in
+    ConvShape("m_is_cin_3x3", 1, 16, 16, 128, 64, 3, 3, 1, 1, 1, 64, 128, 8),         # 50 %, M = C_in, tile 8
+    ConvShape("m_is_row", 1, 12, 12, 64, 64, 3, 3, 1, 1, 1, 144, 576, 16),            # 75 %, M = the whole row K
+    ConvShape("m_64_of_96", 2, 10, 10, 96, 32, 1, 1, 1, 0, 1, 24, 96, 32),
+]
+
+
+@pytest.mark.parametrize("s", LARGE_M, ids=lambda s: s.name)
+def test_large_groups(nm, s):
+    big = s.batch * s.h * s.w * s.c_in * 4 >= 131072
+    _run(nm, s, need_variant=[1] + ([4] if big else []))
+
+
+@pytest.mark.parametrize("s", LARGE_M[:2], ids=lambda s: s.name)
+def test_large_groups_integer_exact(nm, s):
+    _run(nm, s, integer=True)
+
+
 def test_no_bias_no_relu(nm):
     _run(nm, SMALL[0].with_(relu=False), use_bias=False)
 
