@@ -467,7 +467,8 @@ def main():
         by_kernel = {}
         for (s, hnd, x, bias, y, plan), row in zip(state, table):
             k = KERNEL_OF_VARIANT.get(plan.variant, "library default")
-            acc = by_kernel.setdefault(k, {"ms": 0.0, "bytes": 0, "flops": 0, "launches": 0})
+            acc = by_kernel.setdefault(k, {"ms": 0.0, "bytes": 0, "flops": 0, "launches": 0, "roof_ms": 0.0})
+            acc["roof_ms"] += row["ms"] * row["roofline_frac"]
             acc["ms"] += row["ms"]
             acc["bytes"] += algorithmic_bytes(s)
             acc["flops"] += useful_flops(s)
@@ -487,6 +488,7 @@ def main():
             "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],
             "share_of_step": d["ms"] / total_ms,
             "useful_tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12,
+            "time_frac_of_layer_rooflines": d["roof_ms"] / d["ms"],   # some of its layers are tensor-bound, not HBM-bound
             "note": "algorithmic bytes of the layers this kernel runs / their summed launch times (per layer: median of 3 runs "
                     "of >= 20 back-to-back launches on rotating buffers larger than twice the L2)",
         }
