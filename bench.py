@@ -307,7 +307,7 @@ def main():
     ap.add_argument("--bn", type=int, default=0, help="with --variant: output channels per CTA")
     ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
     ap.add_argument("--split", type=int, default=0, help="with --variant: the plan's split field")
-    ap.add_argument("--depth", type=int, default=50, choices=[50, 101, 152], help="ResNet depth of the conv stack")
+    ap.add_argument("--depth", type=int, default=50, choices=[18, 34, 50, 101, 152], help="ResNet depth of the conv stack")
     ap.add_argument("--nm", default="2:4", help="N:M pattern of the pruned layers, e.g. 1:4 or 2:8")
     ap.add_argument("--tile", type=int, default=64, help="pruning tile width T")
     ap.add_argument("--adaptive", type=float, default=None,

@@ -124,14 +124,41 @@ def config_bottleneck1x1():
     return out
 
 
+def _basic_block_stack(depth: int, batch: int, n_keep: int, m_group: int, tile_t: int, image: int):
+    """ResNet-18 / 34 (He et al. 2016): 7x7/2 stem, 3x3/2 max-pool, four stages of basic blocks (two
+    3x3 convolutions; the first one of a stage's first block has stride 2 from stage 2 on, with a
+    1x1/2 projection on its shortcut).  The networks on which the paper reports its largest gains."""
+    blocks = {18: (2, 2, 2, 2), 34: (3, 4, 6, 3)}[depth]
+    layers = [ConvShape("stem7x7", batch, image, image, 3, 64, 7, 7, 2, 3, 1, 1, 1, min(tile_t, 64))]
+    hw = (layers[0].ho + 2 - 3) // 2 + 1   # max-pool -> 56
+    c_prev = 64
+    for si, nb in enumerate(blocks):
+        width = 64 << si
+        for bi in range(nb):
+            stride = 2 if (bi == 0 and si > 0) else 1
+            pre = f"s{si + 1}b{bi + 1}"
+            mk = dict(n_keep=n_keep, m_group=m_group, tile_t=tile_t)
+            layers.append(ConvShape(pre + "_c1", batch, hw, hw, c_prev, width, 3, 3, stride, 1, **mk))
+            hw_out = (hw + 2 - 3) // stride + 1
+            layers.append(ConvShape(pre + "_c2", batch, hw_out, hw_out, width, width, 3, 3, 1, 1, relu=False, **mk))
+            if stride == 2:
+                layers.append(ConvShape(pre + "_ds", batch, hw, hw, c_prev, width, 1, 1, 2, 0, relu=False, **mk))
+            hw = hw_out
+            c_prev = width
+    return layers
+
+
 def resnet_conv_stack(depth: int, batch: int, n_keep: int, m_group: int, tile_t: int = 64, image: int = 224):
-    """Every convolution of a bottleneck ResNet (50 / 101 / 152) in network order.
+    """Every convolution of a ResNet in network order: bottleneck ResNets (50 / 101 / 152) as described
+    below, basic-block ResNets (18 / 34) through ``_basic_block_stack``.
 
     Standard architecture (He et al. 2016): 7x7/2 stem, 3x3/2 max-pool, four stages of
     bottleneck blocks (1x1, 3x3, 1x1; the stride sits on the 3x3 of a stage's first block;
     a 1x1 projection on the first block's shortcut).  The stem keeps every column
     (Sec. 4.1.2: the first convolution is not pruned): it is returned with N = M = 1.
     """
+    if depth in (18, 34):
+        return _basic_block_stack(depth, batch, n_keep, m_group, tile_t, image)
     blocks = {50: (3, 4, 6, 3), 101: (3, 4, 23, 3), 152: (3, 8, 36, 3)}[depth]
     layers = [ConvShape("stem7x7", batch, image, image, 3, 64, 7, 7, 2, 3, 1, 1, 1, min(tile_t, 64))]
     hw = layers[0].ho  # 112

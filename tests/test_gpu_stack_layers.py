@@ -13,7 +13,10 @@ pytestmark = pytest.mark.gpu
 
 # stem (dense, few channels), 1x1 wide output, 3x3 at 56x56, strided 3x3, strided 1x1 projection,
 # tensor-bound 3x3 at 14x14, long-reduction 1x1 and 3x3 at 7x7 (split-K candidates)
-LAYERS = ["stem7x7", "s1b1_c3", "s1b1_c2", "s2b1_c2", "s2b1_ds", "s3b2_c2", "s4b2_c1", "s4b2_c2"]
+LAYERS = [(50, "stem7x7"), (50, "s1b1_c3"), (50, "s1b1_c2"), (50, "s2b1_c2"), (50, "s2b1_ds"), (50, "s3b2_c2"),
+          (50, "s4b2_c1"), (50, "s4b2_c2"),
+          # basic-block network (ResNet-34): strided 3x3 that doubles the channels, 3x3 at 28x28
+          (34, "s2b1_c1"), (34, "s2b2_c2")]
 IMAGES = (0, 37, 63)
 
 
@@ -25,13 +28,13 @@ def nm():
 
 @pytest.fixture(scope="module")
 def stack():
-    layers = inputs.resnet_conv_stack(50, 64, 2, 4, tile_t=64)
-    return {s.name: (i, s) for i, s in enumerate(layers)}
+    return {depth: {s.name: (i, s) for i, s in enumerate(inputs.resnet_conv_stack(depth, 64, 2, 4, tile_t=64))}
+            for depth in (34, 50)}
 
 
-@pytest.mark.parametrize("name", LAYERS)
-def test_stack_layer_sampled_images(nm, stack, name):
-    li, s = stack[name]
+@pytest.mark.parametrize("depth,name", LAYERS, ids=[f"r{d}_{n}" for d, n in LAYERS])
+def test_stack_layer_sampled_images(nm, stack, depth, name):
+    li, s = stack[depth][name]
     w = inputs.make_weights(s, li)
     b = inputs.make_bias(s, li)
     g = torch.Generator().manual_seed(1 + 1000 * li)

@@ -30,3 +30,9 @@ def test_resnet_stacks_have_the_published_conv_counts_and_flops():
     assert r50[0].kk == r50[0].k == 147  # stem keeps every column
     # spatial sizes chain: last block works on 7x7
     assert (r50[-1].ho, r50[-1].c_out) == (7, 2048)
+    # basic-block networks: 1 + 16 + 3 = 20 and 1 + 32 + 3 = 36 convolutions, ~1.8 and ~3.6 GMAC per image
+    r18, r34 = inputs.resnet_conv_stack(18, 1, 2, 4), inputs.resnet_conv_stack(34, 1, 2, 4)
+    assert (len(r18), len(r34)) == (20, 36)
+    assert abs(sum(s.pixels * s.c_out * s.k for s in r18) / 1e9 - 1.81) < 0.05
+    assert abs(sum(s.pixels * s.c_out * s.k for s in r34) / 1e9 - 3.66) < 0.05
+    assert (r34[-1].ho, r34[-1].c_out, r34[-1].kh) == (7, 512, 3)
