@@ -52,6 +52,8 @@ def _load():
         lib.nm_oracle_expand.restype = i
         lib.nm_oracle_conv2d.argtypes = [fp, up] + [i] * 6 + [fp] + [i] * 9 + [fp, i, fp]
         lib.nm_oracle_conv2d.restype = i
+        lib.nm_oracle_conv2d_res.argtypes = [fp, up] + [i] * 6 + [fp] + [i] * 9 + [fp, fp, i, fp]
+        lib.nm_oracle_conv2d_res.restype = i
         _lib = lib
     return _lib
 
@@ -113,6 +115,40 @@ def expand(values: np.ndarray, indices: np.ndarray, k: int, tile_t: int) -> np.n
     if rc != 0:
         raise ValueError("nm_oracle_expand rejected its arguments")
     return out
+
+
+def conv2d_res(values, indices, kh, kw, c_in, tile_t, x, stride=(1, 1), pad=(0, 0), dil=(1, 1),
+               bias=None, residual=None, relu=False) -> np.ndarray:
+    """``conv2d`` followed by the shortcut addition of a residual block before the activation
+    (the block structure of the ResNets measured in Sec. 4.5): ``act(conv + bias + residual)``,
+    the addition in fp64 before the single rounding.  ``residual``: NHWC fp32 of the output's shape."""
+    values, vp = _f32(values)
+    indices, ip = _u16(indices)
+    x, xp = _f32(x)
+    c_out, kk = values.shape
+    b, h, w, ci = x.shape
+    if ci != c_in:
+        raise ValueError("x channel count does not match c_in")
+    ho = (h + 2 * pad[0] - dil[0] * (kh - 1) - 1) // stride[0] + 1
+    wo = (w + 2 * pad[1] - dil[1] * (kw - 1) - 1) // stride[1] + 1
+    y = np.empty((b, ho, wo, c_out), dtype=np.float32)
+    null = ctypes.POINTER(ctypes.c_float)()
+    bp = null
+    if bias is not None:
+        bias, bp = _f32(bias)
+    rp = null
+    if residual is not None:
+        residual, rp = _f32(residual)
+        if residual.shape != y.shape:
+            raise ValueError("residual must have the output's shape")
+    rc = _load().nm_oracle_conv2d_res(
+        vp, ip, c_out, kh, kw, c_in, kk, tile_t, xp, b, h, w,
+        stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], bp, rp, int(bool(relu)),
+        y.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+    )
+    if rc != 0:
+        raise ValueError("nm_oracle_conv2d_res rejected its arguments")
+    return y
 
 
 def conv2d(values, indices, kh, kw, c_in, tile_t, x, stride=(1, 1), pad=(0, 0), dil=(1, 1),

@@ -26,7 +26,9 @@
  * Pins (tests, CPU only): textbook row-wise N:M for T = 1; exhaustive subset search
  * on tiny inputs; hand-worked examples; count/order invariants; N = M identity;
  * zero-expansion round trip; conv against a brute-force 7-loop dense conv, against a
- * library fp64 conv, 1x1 against a plain matrix product, hand-worked 3x3 cases.
+ * library fp64 conv, 1x1 against a plain matrix product, hand-worked 3x3 cases; the
+ * shortcut-adding form against the plain form (zero residual: identical; integer inputs:
+ * exact sum; a library fp64 conv plus the residual).
  */
 #include <math.h>
 #include <stdint.h>
@@ -162,6 +164,55 @@ int nm_oracle_conv2d(const float* values, const uint16_t* indices, int c_out, in
                     }
                     if (relu && acc < 0.0) acc = 0.0;
                     yp[o] = (float)acc;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/*
+ * The same convolution followed by the shortcut addition of a residual block: the networks the
+ * paper measures end to end (Sec. 4.5, torchvision ResNets) add the block input to the last
+ * convolution's output before the ReLU.
+ *   y = act(bias[o] + sum_j values[o][j] * x[...] + residual[n][oh][ow][o])
+ * residual has the output's shape (NHWC fp32) and may be NULL (then this is nm_oracle_conv2d).
+ * Products, the running sum and the shortcut addition in fp64, one rounding to fp32 at the end.
+ */
+int nm_oracle_conv2d_res(const float* values, const uint16_t* indices, int c_out, int kh, int kw,
+                         int c_in, int kk, int tile_t, const float* x, int batch, int h, int w,
+                         int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                         const float* bias, const float* residual, int relu, float* y)
+{
+    if (!values || !indices || !x || !y || c_out < 1 || kh < 1 || kw < 1 || c_in < 1 || kk < 0 ||
+        tile_t < 1 || batch < 1 || h < 1 || w < 1 || stride_h < 1 || stride_w < 1 || pad_h < 0 ||
+        pad_w < 0 || dil_h < 1 || dil_w < 1)
+        return -1;
+    const int ho = (h + 2 * pad_h - dil_h * (kh - 1) - 1) / stride_h + 1;
+    const int wo = (w + 2 * pad_w - dil_w * (kw - 1) - 1) / stride_w + 1;
+    if (h + 2 * pad_h - dil_h * (kh - 1) - 1 < 0 || w + 2 * pad_w - dil_w * (kw - 1) - 1 < 0) return -1;
+
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < batch; ++n) {
+        for (int oh = 0; oh < ho; ++oh) {
+            for (int ow = 0; ow < wo; ++ow) {
+                const size_t pix = ((size_t)n * ho + oh) * wo + ow;
+                for (int o = 0; o < c_out; ++o) {
+                    const uint16_t* idx = indices + (size_t)(o / tile_t) * kk;
+                    const float* val = values + (size_t)o * kk;
+                    double acc = bias ? (double)bias[o] : 0.0;
+                    for (int j = 0; j < kk; ++j) {
+                        const int kcol = idx[j];
+                        const int c = kcol % c_in;
+                        const int tap = kcol / c_in;
+                        const int ih = oh * stride_h - pad_h + (tap / kw) * dil_h;
+                        const int iw = ow * stride_w - pad_w + (tap % kw) * dil_w;
+                        if (ih < 0 || ih >= h || iw < 0 || iw >= w) continue;
+                        acc += (double)val[j] * (double)x[(((size_t)n * h + ih) * w + iw) * c_in + c];
+                    }
+                    if (residual) acc += (double)residual[pix * c_out + o];
+                    if (relu && acc < 0.0) acc = 0.0;
+                    y[pix * c_out + o] = (float)acc;
                 }
             }
         }

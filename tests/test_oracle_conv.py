@@ -174,3 +174,51 @@ def test_rejects_bad_arguments():
         oracle.conv2d(values, indices, 3, 3, 4, 2, x)  # 3x3 on 2x2 without padding: no output
     with pytest.raises(ValueError):
         oracle.conv2d(values, indices, 1, 1, 5, 2, x)  # channel mismatch
+
+
+# ---- shortcut-adding form (residual blocks of the ResNets of Sec. 4.5) -------------------------------
+
+def _res_case(seed=5, integer=False):
+    rng = np.random.default_rng(seed)
+    c_out, kh, kw, c_in = 12, 3, 3, 8
+    if integer:
+        w = rng.integers(-3, 4, (c_out, kh, kw, c_in)).astype(np.float32)
+        x = rng.integers(-3, 4, (2, 7, 6, c_in)).astype(np.float32)
+        b = rng.integers(-3, 4, (c_out,)).astype(np.float32)
+    else:
+        w = rng.standard_normal((c_out, kh, kw, c_in)).astype(np.float32)
+        x = rng.standard_normal((2, 7, 6, c_in)).astype(np.float32)
+        b = rng.standard_normal((c_out,)).astype(np.float32)
+    v, i = oracle.prune(w, 2, 4, 4)
+    return v, i, x, b, (kh, kw, c_in, 4)
+
+
+def test_residual_form_with_zero_or_no_residual_is_the_plain_form():
+    v, i, x, b, (kh, kw, c_in, t) = _res_case()
+    plain = oracle.conv2d(v, i, kh, kw, c_in, t, x, (1, 1), (1, 1), (1, 1), b, True)
+    none = oracle.conv2d_res(v, i, kh, kw, c_in, t, x, (1, 1), (1, 1), (1, 1), b, None, True)
+    zero = oracle.conv2d_res(v, i, kh, kw, c_in, t, x, (1, 1), (1, 1), (1, 1), b, np.zeros_like(plain), True)
+    assert np.array_equal(plain, none) and np.array_equal(plain, zero)
+
+
+def test_residual_is_added_before_the_activation_exactly_on_integers():
+    v, i, x, b, (kh, kw, c_in, t) = _res_case(integer=True)
+    lin = oracle.conv2d(v, i, kh, kw, c_in, t, x, (2, 1), (1, 0), (1, 1), b, False)       # no activation
+    res = np.random.default_rng(9).integers(-20, 21, lin.shape).astype(np.float32)
+    got = oracle.conv2d_res(v, i, kh, kw, c_in, t, x, (2, 1), (1, 0), (1, 1), b, res, True)
+    assert np.array_equal(got, np.maximum(lin + res, 0.0))      # everything is an exact small integer
+    # a ReLU applied before the addition would give something else on this data
+    assert not np.array_equal(got, np.maximum(lin, 0.0) + res)
+
+
+def test_residual_form_equals_library_fp64_conv_plus_residual():
+    torch = pytest.importorskip("torch")
+    v, i, x, b, (kh, kw, c_in, t) = _res_case(seed=11)
+    dense = oracle.expand(v, i, kh * kw * c_in, t).reshape(v.shape[0], kh, kw, c_in)
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).double().permute(0, 3, 1, 2),
+                                     torch.from_numpy(dense).double().permute(0, 3, 1, 2),
+                                     torch.from_numpy(b).double(), stride=1, padding=1).permute(0, 2, 3, 1).numpy()
+    res = np.random.default_rng(3).standard_normal(ref.shape).astype(np.float32)
+    want = np.maximum(ref + res.astype(np.float64), 0.0)
+    got = oracle.conv2d_res(v, i, kh, kw, c_in, t, x, (1, 1), (1, 1), (1, 1), b, res, True)
+    assert np.allclose(got, want, rtol=0, atol=1e-5 * np.abs(want).max())
