@@ -215,6 +215,19 @@ nm_status_t nm_conv2d(const nm_weights_t* w, const float* x, int batch, int h, i
                       void* cuda_stream);
 
 /*
+ * nm_conv2d with the shortcut addition of a residual block fused into the epilogue (the ResNets the
+ * paper measures end to end, Sec. 4.5, add the block input to the last convolution's output before
+ * the ReLU):   y = act(conv(x, W_pruned) + bias + residual)
+ *   residual  device fp32 [batch][ho][wo][c_out] (the output's shape), 16-byte aligned, or NULL
+ *             (then this is nm_conv2d); it may not alias y; needs c_out % 4 == 0
+ * Everything else as nm_conv2d, including the plans.
+ */
+nm_status_t nm_conv2d_res(const nm_weights_t* w, const float* x, int batch, int h, int wd,
+                          int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                          const float* bias, const float* residual, int relu, float* y,
+                          const nm_plan_t* plan, void* cuda_stream);
+
+/*
  * Same operation with HOST buffers: x_host, bias_host and y_host are host pointers (pinned memory
  * makes the copies asynchronous), x_dev / y_dev are caller-owned device staging buffers of the
  * sizes nm_conv2d expects and bias_dev a device buffer of c_out floats (may be NULL iff bias_host

@@ -108,7 +108,7 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     const long long pixels = static_cast<long long>(batch) * ho * wo;
     if (ho > 0x7FFFFFFF || wo > 0x7FFFFFFF || pixels > (1ll << 40))
         return nmhost::fail(NM_ERR_UNSUPPORTED, "%s: output too large", who);
-    p->x = x; p->wt = w->wt; p->taps = w->taps; p->bias = bias; p->y = y; p->status = w->status;
+    p->x = x; p->wt = w->wt; p->taps = w->taps; p->bias = bias; p->residual = nullptr; p->y = y; p->status = w->status;
     p->batch = batch; p->h = h; p->w = wd; p->c_in = w->c_in;
     p->ho = static_cast<int>(ho); p->wo = static_cast<int>(wo); p->c_out = w->c_out;
     p->stride_h = stride_h; p->stride_w = stride_w; p->pad_h = pad_h; p->pad_w = pad_w;
@@ -357,6 +357,22 @@ nm_status_t nm_conv2d(const nm_weights_t* w, const float* x, int batch, int h, i
     nm_status_t s = make_params("nm_conv2d", w, x, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, bias,
                                 relu, y, &p);
     if (s != NM_OK) return s;
+    return run_plan(p, plan, static_cast<cudaStream_t>(cuda_stream));
+}
+
+nm_status_t nm_conv2d_res(const nm_weights_t* w, const float* x, int batch, int h, int wd, int stride_h, int stride_w,
+                          int pad_h, int pad_w, int dil_h, int dil_w, const float* bias, const float* residual,
+                          int relu, float* y, const nm_plan_t* plan, void* cuda_stream)
+{
+    ConvParams p;
+    nm_status_t s = make_params("nm_conv2d_res", w, x, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                bias, relu, y, &p);
+    if (s != NM_OK) return s;
+    if (residual && !aligned16(residual))
+        return nmhost::fail(NM_ERR_INVALID_ARG, "nm_conv2d_res: residual must be 16-byte aligned");
+    if (residual && p.c_out % 4 != 0)
+        return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d_res: c_out must be a multiple of 4");
+    p.residual = residual;
     return run_plan(p, plan, static_cast<cudaStream_t>(cuda_stream));
 }
 

@@ -228,11 +228,13 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 }
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
+                const float4* rrow = nm_residual_row(p, static_cast<long long>(pix0) + q * 32 + lane, o0 + blk * 32);
 #pragma unroll
                 for (int qq = 0; qq < 8; ++qq) {
                     float o[4];
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
+                    if (rrow) nm_add4(bv, __ldg(rrow + qq));
                     o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                     o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                     o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
@@ -271,9 +273,10 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
-// Second pass of a split-K plan: y[p][c] = act(sum over splits of partial[s][p][c] + bias[c]).
+// Second pass of a split-K plan: y[p][c] = act(sum over splits of partial[s][p][c] + bias[c] + residual[p][c]).
 __global__ void k_splitk_reduce(const float4* __restrict__ part, int splits, size_t split_stride4, size_t n4, int c_out4,
-                                const float4* __restrict__ bias, int relu, float4* __restrict__ y)
+                                const float4* __restrict__ bias, const float4* __restrict__ residual, int relu,
+                                float4* __restrict__ y)
 {
     nmk::pdl_wait();   // the partial sums come from the kernel launched just before
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n4;
@@ -285,6 +288,10 @@ __global__ void k_splitk_reduce(const float4* __restrict__ part, int splits, siz
         }
         if (bias) {
             const float4 b = __ldg(bias + (i % c_out4));
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        if (residual) {
+            const float4 b = __ldg(residual + i);
             a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
         }
         if (relu) { a.x = fmaxf(a.x, 0.f); a.y = fmaxf(a.y, 0.f); a.z = fmaxf(a.z, 0.f); a.w = fmaxf(a.w, 0.f); }
@@ -382,6 +389,7 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
         q.y = p.splitk;
         q.pixels = static_cast<long long>(cfg.ksplit) * cfg.p_pad;   // rows of the store map
         q.bias = nullptr;
+        q.residual = nullptr;
         q.relu = 0;
     }
     alignas(64) CUtensorMap tm_x, tm_y;
@@ -405,7 +413,8 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
         if (blocks > static_cast<size_t>(sm_count()) * 8) blocks = static_cast<size_t>(sm_count()) * 8;
         e = nmhost::launch_pdl(k_splitk_reduce, static_cast<unsigned>(blocks), 256u, 0, st,
                                reinterpret_cast<const float4*>(p.splitk), cfg.ksplit, stride4, n4, p.c_out / 4,
-                               reinterpret_cast<const float4*>(p.bias), p.relu, reinterpret_cast<float4*>(p.y));
+                               reinterpret_cast<const float4*>(p.bias), reinterpret_cast<const float4*>(p.residual), p.relu,
+                               reinterpret_cast<float4*>(p.y));
         nmhost::count_launch(1);
         if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (split-K reduction): %s", cudaGetErrorString(e));

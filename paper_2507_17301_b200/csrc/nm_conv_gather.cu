@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(128) k_conv_gather(const ConvParams p, const i
                         for (int e = 0; e < 4; ++e) {
                             float t = __uint_as_float(v[q + e]);
                             if (p.bias) t += __ldg(p.bias + o_base + col0 + q + e);
+                            if (p.residual) t += __ldg(p.residual + (yrow - p.y) + o_base + col0 + q + e);
                             o[e] = p.relu ? fmaxf(t, 0.f) : t;
                         }
                         *reinterpret_cast<float4*>(yrow + o_base + col0 + q) = o4;
@@ -152,6 +153,7 @@ __global__ void __launch_bounds__(128) k_conv_gather(const ConvParams p, const i
                         if (col0 + q < n_valid) {
                             float t = __uint_as_float(v[q]);
                             if (p.bias) t += __ldg(p.bias + o_base + col0 + q);
+                            if (p.residual) t += __ldg(p.residual + (yrow - p.y) + o_base + col0 + q);
                             yrow[o_base + col0 + q] = p.relu ? fmaxf(t, 0.f) : t;
                         }
                     }

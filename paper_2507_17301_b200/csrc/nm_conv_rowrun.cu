@@ -222,11 +222,15 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                 if (lane == 0 && nb >= 2) tma_store_wait_read_n<1>();
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
+                // pixel of this thread: output row `work`, column q * 32 + lane (past the row's end: none)
+                const float4* rrow = nm_residual_row(
+                    p, q * 32 + lane < p.wo ? static_cast<long long>(work) * p.wo + q * 32 + lane : p.pixels, blk * 32);
 #pragma unroll
                 for (int qq = 0; qq < 8; ++qq) {
                     float o[4];
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + blk * 32) + qq);
+                    if (rrow) nm_add4(bv, __ldg(rrow + qq));
                     o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                     o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                     o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;

@@ -256,11 +256,13 @@ k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUten
                     tmem_ld32(tmem + lane_addr + blk * 32, v);
                     tmem_ld_wait();
                     const uint32_t stage_row = ring + blk * SUB_BYTES + row * 128;
+                    const float4* rrow = nm_residual_row(p, pix0 + row, o0 + blk * 32);
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
                         float o[4];
                         float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                         if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + q);
+                        if (rrow) nm_add4(bv, __ldg(rrow + q));
                         o[0] = __uint_as_float(v[q * 4 + 0]) + bv.x;
                         o[1] = __uint_as_float(v[q * 4 + 1]) + bv.y;
                         o[2] = __uint_as_float(v[q * 4 + 2]) + bv.z;
@@ -306,6 +308,7 @@ k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUten
                                 for (int e = 0; e < 4; ++e) {
                                     float tt = __uint_as_float(v[q + e]);
                                     if (p.bias) tt += __ldg(p.bias + o_base + col0 + q + e);
+                                    if (p.residual) tt += __ldg(p.residual + (yrow - p.y) + o_base + col0 + q + e);
                                     o[e] = p.relu ? fmaxf(tt, 0.f) : tt;
                                 }
                                 *reinterpret_cast<float4*>(yrow + o_base + col0 + q) = o4;
@@ -316,6 +319,7 @@ k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUten
                                 if (col0 + q < n_valid) {
                                     float tt = __uint_as_float(v[q]);
                                     if (p.bias) tt += __ldg(p.bias + o_base + col0 + q);
+                                    if (p.residual) tt += __ldg(p.residual + (yrow - p.y) + o_base + col0 + q);
                                     yrow[o_base + col0 + q] = p.relu ? fmaxf(tt, 0.f) : tt;
                                 }
                             }

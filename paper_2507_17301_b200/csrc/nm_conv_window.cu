@@ -261,6 +261,8 @@ k_conv_window(const ConvParams p, const WinCfg cfg, const __grid_constant__ CUte
                             float4 o;
                             float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                             if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
+                            if (p.residual)
+                                nm_add4(bv, __ldg(reinterpret_cast<const float4*>(p.residual + (yrow - p.y) + blk * 32 + qq * 4)));
                             o.x = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                             o.y = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                             o.z = __uint_as_float(v[qq * 4 + 2]) + bv.z;

@@ -39,6 +39,7 @@ struct ConvParams {
     const float* wt;
     const uint32_t* taps;
     const float* bias;
+    const float* residual;   // shortcut input added before the activation: the output's shape, or NULL
     float* y;
     int* status;
     int batch, h, w, c_in, ho, wo, c_out;
@@ -58,6 +59,19 @@ struct ConvParams {
     float* splitk;
     size_t splitk_bytes;
 };
+
+#ifdef __CUDACC__
+// Shortcut input of one output pixel from channel `channel` on, as float4s (NULL without a residual or past the end).
+__device__ __forceinline__ const float4* nm_residual_row(const ConvParams& p, long long pixel, int channel)
+{
+    if (!p.residual || pixel >= p.pixels) return nullptr;
+    return reinterpret_cast<const float4*>(p.residual + pixel * p.c_out + channel);
+}
+__device__ __forceinline__ void nm_add4(float4& a, const float4& b)
+{
+    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+}
+#endif
 
 namespace nmhost {
 // Launches `kernel` so that it may begin while the previous kernel of the stream drains

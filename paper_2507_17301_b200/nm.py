@@ -58,6 +58,8 @@ def _load():
     lib.nm_weights_free.argtypes = [vp]
     conv_geom = [i] * 9
     lib.nm_conv2d.argtypes = [vp, vp] + conv_geom + [vp, i, vp, pp, vp]
+    lib.nm_conv2d_res.argtypes = [vp, vp] + conv_geom + [vp, vp, i, vp, pp, vp]
+    lib.nm_conv2d_res.restype = ctypes.c_int
     lib.nm_conv2d_host.argtypes = [vp, vp, vp] + conv_geom + [vp, vp, i, vp, vp, pp, vp]
     lib.nm_autotune.argtypes = [vp, vp] + conv_geom + [vp, i, vp, vp, pp, fp]
     lib.nm_autotune_tile.argtypes = [vp, i, i, i, i, i, i, ip, i, vp] + conv_geom + [vp, i, vp, vp, ip, pp, fp]
@@ -77,7 +79,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -216,8 +218,10 @@ def out_shape(x_shape, kh, kw, c_out, stride, pad, dil):
 
 
 def nm_conv2d(w: Weights, x: torch.Tensor, kh: int, kw: int, stride=1, pad=0, dil=1, bias=None, relu=False,
-              y: torch.Tensor | None = None, plan: nm_plan_t | None = None) -> torch.Tensor:
-    """``x``: CUDA fp32 NHWC.  Allocates ``y`` (NHWC) unless given.  Asynchronous on the current stream."""
+              y: torch.Tensor | None = None, plan: nm_plan_t | None = None,
+              residual: torch.Tensor | None = None) -> torch.Tensor:
+    """``x``: CUDA fp32 NHWC.  Allocates ``y`` (NHWC) unless given.  Asynchronous on the current stream.
+    With ``residual`` (NHWC, the output's shape) it calls ``nm_conv2d_res``: act(conv + bias + residual)."""
     stride, pad, dil = _pair(stride), _pair(pad), _pair(dil)
     xp = _dev_f32(x, "x")
     b, h, wd, _ = x.shape
@@ -229,8 +233,15 @@ def nm_conv2d(w: Weights, x: torch.Tensor, kh: int, kw: int, stride=1, pad=0, di
             y = torch.empty([max(d, 1) for d in shape], dtype=torch.float32, device=x.device)
     yp = _dev_f32(y, "y")
     bp = _dev_f32(bias, "bias") if bias is not None else None
-    _check(_lib.nm_conv2d(w.handle, xp, b, h, wd, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], bp,
-                          int(bool(relu)), yp, ctypes.byref(plan) if plan is not None else None, _stream()))
+    pl = ctypes.byref(plan) if plan is not None else None
+    if residual is None:
+        _check(_lib.nm_conv2d(w.handle, xp, b, h, wd, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], bp,
+                              int(bool(relu)), yp, pl, _stream()))
+    else:
+        if tuple(residual.shape) != tuple(y.shape):
+            raise TypeError("residual must have the output's shape")
+        _check(_lib.nm_conv2d_res(w.handle, xp, b, h, wd, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], bp,
+                                  _dev_f32(residual, "residual"), int(bool(relu)), yp, pl, _stream()))
     return y
 
 
