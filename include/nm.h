@@ -147,6 +147,14 @@ nm_status_t nm_weights_dims(const nm_weights_t* w, int* c_out, int* k, int* kk, 
                             int* tile_t);
 
 /*
+ * L1 mass of the retained weights and of all weights of the layer (sums of |w|, fp64): kept / total is
+ * the share of the importance measure of Sec. 3.1 that survived pruning, the accuracy proxy to read
+ * next to a tile width (wider tiles share a kept set among more rows and retain less).  Known only
+ * for handles made by nm_prune (NM_ERR_UNSUPPORTED for imported ones).  Either pointer may be NULL.
+ */
+nm_status_t nm_weights_retained_l1(const nm_weights_t* w, double* kept, double* total);
+
+/*
  * Copies the canonical compressed form (the compacted weights plus index array of Sec. 2.1,
  * i.e. Algorithm 1's inputs W[T, N] and Idx[N]) to caller memory on `cuda_stream`:
  *   values   device, fp32 [c_out][kk]: values[o][j] = w[o][indices[o / tile_t][j]], bit-exact

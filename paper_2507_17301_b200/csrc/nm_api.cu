@@ -63,6 +63,8 @@ nm_status_t make_handle(const char* who, int c_out, int kh, int kw, int c_in, in
     if (!h) return nmhost::fail(NM_ERR_ALLOC, "%s: out of host memory", who);
     std::memset(h, 0, sizeof(*h));
     h->magic = NM_MAGIC;
+    h->l1_total = -1.0;
+    h->l1_kept = -1.0;
     h->device = dev;
     h->c_out = c_out; h->kh = kh; h->kw = kw; h->c_in = c_in;
     h->k = static_cast<int>(k);
@@ -275,6 +277,16 @@ nm_status_t nm_weights_dims(const nm_weights_t* w, int* c_out, int* k, int* kk, 
     if (kk) *kk = w->kk;
     if (n_tiles) *n_tiles = w->n_tiles;
     if (tile_t) *tile_t = w->tile_t;
+    return NM_OK;
+}
+
+nm_status_t nm_weights_retained_l1(const nm_weights_t* w, double* kept, double* total)
+{
+    if (!valid(w)) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_weights_retained_l1: bad weights handle");
+    if (w->l1_total < 0.0)
+        return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_weights_retained_l1: the handle was imported, the dense weights were never seen");
+    if (kept) *kept = w->l1_kept;
+    if (total) *total = w->l1_total;
     return NM_OK;
 }
 

@@ -16,6 +16,7 @@ struct nm_weights {
     int device;
     int c_out, kh, kw, c_in, k, kk, n_keep, m_group, tile_t, n_tiles;
     int kk_pad;          // kk rounded up to a multiple of NM_KCHUNK
+    double l1_total, l1_kept;   // L1 mass of the dense weights / of the retained ones (l1_total < 0: not known)
     float* values;       // [c_out][kk]     exact fp32 copies of the retained weights
     uint16_t* indices;   // [n_tiles][kk]   retained column positions, ascending
     float* wt;           // [c_out][kk_pad] retained weights rounded to TF32 (nearest), zero padded

@@ -48,6 +48,27 @@ __global__ void k_select(const double* __restrict__ score, int k, int n_keep, in
     keep[static_cast<size_t>(r) * k + col] = beaten_by < n_keep ? 1 : 0;
 }
 
+// L1 mass of all columns and of the retained ones: mass[0] += score, mass[1] += score * keep.
+__global__ void k_mass(const double* __restrict__ score, const uint8_t* __restrict__ keep, size_t cells,
+                       double* __restrict__ mass)
+{
+    double all = 0.0, kept = 0.0;
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < cells;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const double s = score[i];
+        all += s;
+        if (keep[i]) kept += s;
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        all += __shfl_down_sync(0xFFFFFFFFu, all, d);
+        kept += __shfl_down_sync(0xFFFFFFFFu, kept, d);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(mass + 0, all);
+        atomicAdd(mass + 1, kept);
+    }
+}
+
 __global__ void k_compact(const uint8_t* __restrict__ keep, int k, int kk, int kk_pad, int n_keep, int m_group,
                           int c_in, int kw, uint16_t* __restrict__ indices, uint32_t* __restrict__ taps)
 {
@@ -163,6 +184,7 @@ nm_status_t prune_on_device(const float* w_dense, nm_weights* h, cudaStream_t st
 {
     nm_status_t st_out = NM_OK;
     double* score = nullptr;
+    double* mass = nullptr;
     uint8_t* keep = nullptr;
     const size_t cells = static_cast<size_t>(h->n_tiles) * h->k;
     const dim3 blk(128);
@@ -183,10 +205,25 @@ nm_status_t prune_on_device(const float* w_dense, nm_weights* h, cudaStream_t st
                                                h->wt);
     count_launch(4);
     NM_CUDA_TRY(cudaGetLastError());
-    NM_CUDA_TRY(cudaStreamSynchronize(st));  // the scratch is freed below
+    {
+        // retained share of the L1 mass (the accuracy proxy reported next to a tile width)
+        double host_mass[2] = {0.0, 0.0};
+        NM_CUDA_TRY(cudaMalloc(&mass, 2 * sizeof(double)));
+        NM_CUDA_TRY(cudaMemsetAsync(mass, 0, 2 * sizeof(double), st));
+        size_t blocks = (cells + 255) / 256;
+        if (blocks > 1024) blocks = 1024;
+        k_mass<<<static_cast<unsigned>(blocks), 256, 0, st>>>(score, keep, cells, mass);
+        count_launch(1);
+        NM_CUDA_TRY(cudaGetLastError());
+        NM_CUDA_TRY(cudaMemcpyAsync(host_mass, mass, sizeof(host_mass), cudaMemcpyDeviceToHost, st));
+        NM_CUDA_TRY(cudaStreamSynchronize(st));  // also: the scratch is freed below
+        h->l1_total = host_mass[0];
+        h->l1_kept = host_mass[1];
+    }
 done:
     cudaFree(score);
     cudaFree(keep);
+    cudaFree(mass);
     return st_out;
 }
 

@@ -53,6 +53,8 @@ def _load():
     lib.nm_weights_export.argtypes = [vp, vp, vp, vp]
     lib.nm_weights_import.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, ctypes.POINTER(vp)]
     lib.nm_weights_check.argtypes = [vp, vp]
+    lib.nm_weights_retained_l1.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    lib.nm_weights_retained_l1.restype = ctypes.c_int
     lib.nm_plan_scratch_bytes.argtypes = [vp] + [i] * 9 + [pp, ctypes.POINTER(ctypes.c_size_t)]
     lib.nm_weights_reserve.argtypes = [vp, ctypes.c_size_t]
     lib.nm_weights_free.argtypes = [vp]
@@ -79,7 +81,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -204,6 +206,13 @@ def nm_plan_scratch_bytes(w: Weights, x_shape, stride, pad, dil, plan: nm_plan_t
 def nm_weights_reserve(w: Weights, nbytes: int):
     """Reserves handle-owned scratch memory (allocates; call outside the timed / captured region)."""
     _check(_lib.nm_weights_reserve(w.handle, nbytes))
+
+
+def nm_weights_retained_l1(w: Weights):
+    """Returns ``(kept, total)``: L1 mass of the retained weights and of all weights of the layer."""
+    kept, total = ctypes.c_double(), ctypes.c_double()
+    _check(_lib.nm_weights_retained_l1(w.handle, ctypes.byref(kept), ctypes.byref(total)))
+    return float(kept.value), float(total.value)
 
 
 def nm_weights_check(w: Weights):

@@ -80,3 +80,26 @@ def test_import_round_trip_and_validation(nm):
     with pytest.raises(nm.NmError) as e:
         nm.nm_weights_import(v, bad.view(torch.uint16), 3, 3, 16, 2, 4, 8)
     assert e.value.status == nm.NM_ERR_INVALID_ARG
+
+
+
+def test_retained_l1_mass(nm):
+    """Retained / total L1 mass against the plain sums over the oracle's result; wider tiles retain less."""
+    import numpy as np
+    import oracle
+    g = torch.Generator().manual_seed(5)
+    w = torch.randn((96, 3, 3, 32), generator=g)
+    shares = []
+    for t in (1, 8, 32, 96):
+        hnd = nm.nm_prune(w.cuda(), 2, 4, t)
+        kept, total = nm.nm_weights_retained_l1(hnd)
+        vr, _ = oracle.prune(w.numpy(), 2, 4, t)
+        assert total == pytest.approx(float(np.abs(w.numpy().astype(np.float64)).sum()), rel=1e-9)
+        assert kept == pytest.approx(float(np.abs(vr.astype(np.float64)).sum()), rel=1e-9)
+        shares.append(kept / total)
+    assert shares == sorted(shares, reverse=True) and shares[0] > shares[-1]
+    v, i = nm.nm_weights_export(nm.nm_prune(w.cuda(), 2, 4, 32))
+    imported = nm.nm_weights_import(v, i, 3, 3, 32, 2, 4, 32)
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_weights_retained_l1(imported)
+    assert e.value.status == nm.NM_ERR_UNSUPPORTED
