@@ -246,6 +246,18 @@ nm_status_t nm_conv2d_host(const nm_weights_t* w, const float* x_host, float* x_
                            int dil_h, int dil_w, const float* bias_host, float* bias_dev, int relu,
                            float* y_host, float* y_dev, const nm_plan_t* plan, void* cuda_stream);
 
+/*
+ * Max pooling over NHWC fp32 activations (the paper has no counterpart in its method: it is the one
+ * layer between the stem and the first residual block of the ResNets of Sec. 4.5, provided so that a
+ * whole convolution backbone can run through this library):
+ *   y[n][oh][ow][ch] = max over the kh x kw window at (oh*stride_h - pad_h, ow*stride_w - pad_w) of x,
+ * window positions outside the image ignored; ho = (h + 2*pad_h - kh) / stride_h + 1 (floor), wo alike.
+ *   x  device fp32 [batch][h][w][c]      y  device fp32 [batch][ho][wo][c]      c % 4 == 0, pad < window
+ * Asynchronous on `cuda_stream`; allocates nothing.
+ */
+nm_status_t nm_maxpool2d(const float* x, int batch, int h, int w, int c, int kh, int kw, int stride_h,
+                         int stride_w, int pad_h, int pad_w, float* y, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Auto-tuning (Sec. 3.3: profile kernel candidates on the target, keep the fastest)
  * ------------------------------------------------------------------------------------------- */

@@ -54,6 +54,8 @@ def _load():
         lib.nm_oracle_conv2d.restype = i
         lib.nm_oracle_conv2d_res.argtypes = [fp, up] + [i] * 6 + [fp] + [i] * 9 + [fp, fp, i, fp]
         lib.nm_oracle_conv2d_res.restype = i
+        lib.nm_oracle_maxpool2d.argtypes = [fp] + [i] * 10 + [fp]
+        lib.nm_oracle_maxpool2d.restype = i
         _lib = lib
     return _lib
 
@@ -179,4 +181,21 @@ def conv2d(values, indices, kh, kw, c_in, tile_t, x, stride=(1, 1), pad=(0, 0), 
     )
     if rc != 0:
         raise ValueError("nm_oracle_conv2d rejected its arguments")
+    return y
+
+
+def maxpool2d(x, kernel=(3, 3), stride=(2, 2), pad=(1, 1)) -> np.ndarray:
+    """Max pooling over NHWC fp32 (between the stem and the first block of the ResNets of Sec. 4.5);
+    window positions outside the image do not take part."""
+    x, xp = _f32(x)
+    b, h, w, c = x.shape
+    ho = (h + 2 * pad[0] - kernel[0]) // stride[0] + 1
+    wo = (w + 2 * pad[1] - kernel[1]) // stride[1] + 1
+    if ho < 1 or wo < 1:
+        raise ValueError("the window does not fit the padded image")
+    y = np.empty((b, ho, wo, c), dtype=np.float32)
+    rc = _load().nm_oracle_maxpool2d(xp, b, h, w, c, kernel[0], kernel[1], stride[0], stride[1], pad[0], pad[1],
+                                     y.ctypes.data_as(ctypes.POINTER(ctypes.c_float)))
+    if rc != 0:
+        raise ValueError("nm_oracle_maxpool2d rejected its arguments")
     return y

@@ -219,3 +219,36 @@ int nm_oracle_conv2d_res(const float* values, const uint16_t* indices, int c_out
     }
     return 0;
 }
+
+/*
+ * Max pooling over NHWC fp32 (the layer between the stem and the first residual block of the
+ * ResNets of Sec. 4.5): y[n][oh][ow][c] = max of x over the kh x kw window whose corner is
+ * (oh*stride_h - pad_h, ow*stride_w - pad_w); positions outside the image do not take part.
+ * Returns 0, -1 on a bad argument (padding must be smaller than the window).
+ */
+int nm_oracle_maxpool2d(const float* x, int batch, int h, int w, int c, int kh, int kw, int stride_h,
+                        int stride_w, int pad_h, int pad_w, float* y)
+{
+    if (!x || !y || batch < 1 || h < 1 || w < 1 || c < 1 || kh < 1 || kw < 1 || stride_h < 1 ||
+        stride_w < 1 || pad_h < 0 || pad_w < 0 || pad_h >= kh || pad_w >= kw || h + 2 * pad_h < kh ||
+        w + 2 * pad_w < kw)
+        return -1;
+    const int ho = (h + 2 * pad_h - kh) / stride_h + 1, wo = (w + 2 * pad_w - kw) / stride_w + 1;
+    for (int n = 0; n < batch; ++n)
+        for (int oh = 0; oh < ho; ++oh)
+            for (int ow = 0; ow < wo; ++ow)
+                for (int ch = 0; ch < c; ++ch) {
+                    int seen = 0;
+                    float m = 0.0f;
+                    for (int i = 0; i < kh; ++i)
+                        for (int j = 0; j < kw; ++j) {
+                            const int ih = oh * stride_h - pad_h + i, iw = ow * stride_w - pad_w + j;
+                            if (ih < 0 || ih >= h || iw < 0 || iw >= w) continue;
+                            const float v = x[(((size_t)n * h + ih) * w + iw) * c + ch];
+                            if (!seen || v > m) m = v;
+                            seen = 1;
+                        }
+                    y[(((size_t)n * ho + oh) * wo + ow) * c + ch] = m;
+                }
+    return 0;
+}

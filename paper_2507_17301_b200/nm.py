@@ -53,6 +53,8 @@ def _load():
     lib.nm_weights_export.argtypes = [vp, vp, vp, vp]
     lib.nm_weights_import.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, ctypes.POINTER(vp)]
     lib.nm_weights_check.argtypes = [vp, vp]
+    lib.nm_maxpool2d.argtypes = [vp] + [i] * 10 + [vp, vp]
+    lib.nm_maxpool2d.restype = ctypes.c_int
     lib.nm_weights_retained_l1.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.nm_weights_retained_l1.restype = ctypes.c_int
     lib.nm_plan_scratch_bytes.argtypes = [vp] + [i] * 9 + [pp, ctypes.POINTER(ctypes.c_size_t)]
@@ -81,7 +83,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_maxpool2d", "nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -206,6 +208,19 @@ def nm_plan_scratch_bytes(w: Weights, x_shape, stride, pad, dil, plan: nm_plan_t
 def nm_weights_reserve(w: Weights, nbytes: int):
     """Reserves handle-owned scratch memory (allocates; call outside the timed / captured region)."""
     _check(_lib.nm_weights_reserve(w.handle, nbytes))
+
+
+def nm_maxpool2d(x: torch.Tensor, kernel=3, stride=2, pad=1, y: torch.Tensor | None = None) -> torch.Tensor:
+    """Max pooling of CUDA fp32 NHWC activations; allocates ``y`` unless given."""
+    kernel, stride, pad = _pair(kernel), _pair(stride), _pair(pad)
+    b, h, wd, c = x.shape
+    if y is None:
+        ho = (h + 2 * pad[0] - kernel[0]) // stride[0] + 1
+        wo = (wd + 2 * pad[1] - kernel[1]) // stride[1] + 1
+        y = torch.empty((b, max(ho, 1), max(wo, 1), c), dtype=torch.float32, device=x.device)
+    _check(_lib.nm_maxpool2d(_dev_f32(x, "x"), b, h, wd, c, kernel[0], kernel[1], stride[0], stride[1], pad[0], pad[1],
+                             _dev_f32(y, "y"), _stream()))
+    return y
 
 
 def nm_weights_retained_l1(w: Weights):
