@@ -521,6 +521,50 @@ def main():
                                   "useful_tflops": flops_step / (g_ms * 1e-3) / 1e12,
                                   "note": "plans restricted to the gathering kernels (variants 1-3)"}
 
+        # the same layers chained as the network's dataflow: stem -> max-pool -> residual blocks, every
+        # layer reading its predecessor's output, shortcut additions fused into the last conv of a block
+        if not args.layer:
+            idx = {s.name: i for i, (s, *_rest) in enumerate(state)}
+            pool_out = torch.empty((args.batch, state[1][0].h, state[1][0].w, 64), dtype=torch.float32, device=dev)
+            prefixes = []
+            for s, *_rest in state[1:]:
+                pre = s.name.rsplit("_", 1)[0]
+                if pre not in prefixes:
+                    prefixes.append(pre)
+
+            def conv(i, x_in, relu, residual=None):
+                s, hnd, _x, bias, y, plan = state[i]
+                nm.nm_conv2d(hnd, x_in, s.kh, s.kw, s.stride, s.pad, s.dil, bias, relu, y=y, plan=plan, residual=residual)
+                return y
+
+            def chained_step():
+                cur = conv(0, state[0][2], True)
+                cur = nm.nm_maxpool2d(cur, 3, 2, 1, y=pool_out)
+                for pre in prefixes:
+                    shortcut = conv(idx[pre + "_ds"], cur, False) if pre + "_ds" in idx else cur
+                    t = conv(idx[pre + "_c1"], cur, True)
+                    if pre + "_c3" in idx:                       # bottleneck block
+                        t = conv(idx[pre + "_c2"], t, True)
+                        cur = conv(idx[pre + "_c3"], t, True, residual=shortcut)
+                    else:                                        # basic block
+                        cur = conv(idx[pre + "_c2"], t, True, residual=shortcut)
+                return cur
+
+            for _ in range(3):
+                last = chained_step()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+            a.record()
+            for _ in range(args.steps):
+                chained_step()
+            b.record()
+            b.synchronize()
+            c_ms = a.elapsed_time(b) / args.steps
+            out["chained"] = {"value": args.batch / (c_ms * 1e-3), "unit": UNIT, "ms_per_step": c_ms,
+                              "finite": bool(torch.isfinite(last).all()),
+                              "note": "conv backbone in dataflow order: stem, 3x3/2 max-pool, residual blocks with the "
+                                      "shortcut addition fused into the block's last convolution"}
+
         # cuDNN dense convolution on the same shapes (context, unpruned weights, TF32 allowed)
         try:
             torch.backends.cudnn.allow_tf32 = True

@@ -76,3 +76,29 @@ def test_residual_argument_errors(nm):
     with pytest.raises(nm.NmError) as e:
         nm.nm_conv2d(hnd, x.cuda(), s.kh, s.kw, s.stride, s.pad, s.dil, b.cuda(), True, residual=bad)
     assert e.value.status == nm.NM_ERR_INVALID_ARG
+
+
+def test_chained_block_matches_oracle_chain(nm):
+    """A small residual block chained on the device (conv -> max-pool -> 1x1 -> 3x3 -> 1x1 + shortcut) against the
+    same chain of oracle calls: each layer consumes the previous layer's device output."""
+    g = torch.Generator().manual_seed(17)
+    x = torch.randn((2, 32, 32, 3), generator=g)
+    ws = [torch.randn(sh, generator=g) * sc for sh, sc in (((64, 7, 7, 3), 0.08), ((32, 1, 1, 64), 0.15),
+                                                            ((32, 3, 3, 32), 0.08), ((64, 1, 1, 32), 0.2))]
+    nms = [(1, 1, 64), (2, 4, 32), (2, 4, 32), (2, 4, 32)]
+    hs = [nm.nm_prune(w.cuda(), n, m, t) for w, (n, m, t) in zip(ws, nms)]
+    pr = [oracle.prune(w.numpy(), n, m, t) for w, (n, m, t) in zip(ws, nms)]
+    # device chain
+    a = nm.nm_conv2d(hs[0], x.cuda(), 7, 7, 2, 3, 1, None, True)
+    p0 = nm.nm_maxpool2d(a, 3, 2, 1)
+    t = nm.nm_conv2d(hs[1], p0, 1, 1, 1, 0, 1, None, True)
+    t = nm.nm_conv2d(hs[2], t, 3, 3, 1, 1, 1, None, True)
+    out = nm.nm_conv2d(hs[3], t, 1, 1, 1, 0, 1, None, True, residual=p0)
+    torch.cuda.synchronize()
+    # oracle chain
+    ra = oracle.conv2d(pr[0][0], pr[0][1], 7, 7, 3, 64, x.numpy(), (2, 2), (3, 3), (1, 1), None, True)
+    rp = oracle.maxpool2d(ra, (3, 3), (2, 2), (1, 1))
+    rt = oracle.conv2d(pr[1][0], pr[1][1], 1, 1, 64, 32, rp, (1, 1), (0, 0), (1, 1), None, True)
+    rt = oracle.conv2d(pr[2][0], pr[2][1], 3, 3, 32, 32, rt, (1, 1), (1, 1), (1, 1), None, True)
+    ro = oracle.conv2d_res(pr[3][0], pr[3][1], 1, 1, 32, 32, rt, (1, 1), (0, 0), (1, 1), None, rp, True)
+    assert_conv_close(out.cpu().numpy(), ro)
