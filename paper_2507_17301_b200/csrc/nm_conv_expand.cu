@@ -206,6 +206,14 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
             const uint32_t pix0 = (rest / static_cast<uint32_t>(cfg.ksplit)) * BM;
             const int ab = static_cast<int>(ti & 1u);
+            // the shortcut input does not depend on the accumulator: its first box is requested before the
+            // wait for the main loop, every later box while the one before it is being stored
+            const long long box_pix = static_cast<long long>(pix0) + q * 32;
+            const bool res_pass = p.residual != nullptr && box_pix < p.pixels;
+            const int res_rows = p.pixels - box_pix < 32 ? static_cast<int>(p.pixels - box_pix) : 32;
+            const float* res_base = res_pass ? p.residual + box_pix * p.c_out + slice * cfg.bn : nullptr;
+            float4 rv[8];
+            if (res_pass && half < n_blk) load_residual_box(rv, res_base + half * 32, p.c_out, res_rows, lane);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
@@ -228,24 +236,29 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 }
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
-                const float4* rrow = nm_residual_row(p, static_cast<long long>(pix0) + q * 32 + lane, o0 + blk * 32);
+                // with a shortcut input the activation waits for the second pass below
+                const int relu_now = res_pass ? 0 : p.relu;
 #pragma unroll
                 for (int qq = 0; qq < 8; ++qq) {
                     float o[4];
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
-                    if (rrow) nm_add4(bv, __ldg(rrow + qq));
                     o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                     o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                     o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
                     o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
-                    if (p.relu) {
+                    if (relu_now) {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
                     }
                     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage_row + ((qq ^ rx) << 4)), "f"(o[0]),
                                  "f"(o[1]), "f"(o[2]), "f"(o[3])
                                  : "memory");
+                }
+                if (res_pass) {
+                    __syncwarp();
+                    apply_residual_box(box, rv, p.relu, lane);
+                    if (blk + 2 < n_blk) load_residual_box(rv, res_base + (blk + 2) * 32, p.c_out, res_rows, lane);
                 }
                 fence_proxy_async();
                 __syncwarp();

@@ -292,24 +292,32 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                 if (lane == 0 && nb >= 2) tma_store_wait_read_n<1>();  // the box's previous store has read it
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
-                const float4* rrow = nm_residual_row(p, static_cast<long long>(pix0) + q * 32 + lane, o0 + blk * 32);
+                // with a shortcut input the activation waits for the second pass below
+                const long long box_pix = static_cast<long long>(pix0) + q * 32;
+                const bool res_pass = p.residual != nullptr && box_pix < p.pixels;
+                const int relu_now = res_pass ? 0 : p.relu;
 #pragma unroll
                 for (int qq = 0; qq < 8; ++qq) {
                     float o[4];
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
-                    if (rrow) nm_add4(bv, __ldg(rrow + qq));
                     o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                     o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                     o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
                     o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
-                    if (p.relu) {
+                    if (relu_now) {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
                     }
                     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage_row + ((qq ^ rx) << 4)), "f"(o[0]),
                                  "f"(o[1]), "f"(o[2]), "f"(o[3])
                                  : "memory");
+                }
+                if (res_pass) {
+                    __syncwarp();
+                    const long long left = p.pixels - box_pix;
+                    add_residual_box(box, p.residual + box_pix * p.c_out + o0 + blk * 32, p.c_out,
+                                     left < 32 ? static_cast<int>(left) : 32, p.relu, lane);
                 }
                 fence_proxy_async();
                 __syncwarp();

@@ -189,6 +189,46 @@ __device__ __forceinline__ void tma_prefetch_desc(const void* tmap)
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
 
+// Adds the shortcut input to a staged 32-pixel x 32-channel output box (128-byte-swizzled rows) and
+// applies the activation, one warp per box.  The lanes walk the box four rows at a time, eight
+// 16-byte pieces per row, so that every global load instruction reads four full 128-byte lines of
+// the residual (a thread reading its own row piece by piece would touch 32 lines per instruction).
+//   res       first residual element of the box's first row; row pitch c_out floats
+//   rows      rows of the box that exist (the last block of a layer may be ragged)
+__device__ __forceinline__ void load_residual_box(float4 (&rv)[8], const float* res, int c_out, int rows, int lane)
+{
+    const int piece = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = i * 4 + (lane >> 3);
+        rv[i] = r < rows ? __ldg(reinterpret_cast<const float4*>(res + static_cast<size_t>(r) * c_out) + piece)
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+__device__ __forceinline__ void apply_residual_box(uint32_t box, const float4 (&rv)[8], int relu, int lane)
+{
+    const int piece = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = i * 4 + (lane >> 3);
+        const uint32_t addr = box + r * 128 + ((static_cast<uint32_t>(piece) ^ static_cast<uint32_t>(r & 7)) << 4);
+        float4 v;
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+        v.x += rv[i].x; v.y += rv[i].y; v.z += rv[i].z; v.w += rv[i].w;
+        if (relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+    }
+}
+// Both steps at once (the loads first: the shared-memory accesses are ordered asm statements and would
+// otherwise serialise them).  Kernels that can afford the registers call the two halves apart, with
+// the loads issued a box ahead.
+__device__ __forceinline__ void add_residual_box(uint32_t box, const float* res, int c_out, int rows, int relu, int lane)
+{
+    float4 rv[8];
+    load_residual_box(rv, res, c_out, rows, lane);
+    apply_residual_box(box, rv, relu, lane);
+}
+
 // ---- tensor memory ---------------------------------------------------------------------------------
 // Executed by one full warp. `ncols` is a power of two in [32, 512]; the base address is written
 // to the shared-memory word `slot`.
