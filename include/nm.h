@@ -293,6 +293,15 @@ nm_status_t nm_autotune_tile(const float* w_dense, int c_out, int kh, int kw, in
  * Diagnostics
  * ------------------------------------------------------------------------------------------- */
 
+/*
+ * Self-test of the failure path: launches one small block that waits, with a budget of a few thousand
+ * polls, on a barrier nothing will ever complete.  The wait runs out, the block records NM_ERR_TIMEOUT
+ * in the handle's status word the way the convolution kernels do and returns normally; the next
+ * nm_weights_check(w) reports NM_ERR_TIMEOUT and clears it, and the context stays usable.  Nothing
+ * faults, traps or hangs.
+ */
+nm_status_t nm_selftest_wait_expiry(const nm_weights_t* w, void* cuda_stream);
+
 const char* nm_status_string(nm_status_t s);
 /* Text of the calling thread's most recent failure ("" if none). Valid until its next failure. */
 const char* nm_last_error(void);

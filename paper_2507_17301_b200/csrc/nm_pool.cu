@@ -36,7 +36,37 @@ __global__ void k_maxpool(const float4* __restrict__ x, int h, int w, int c4, in
     }
 }
 
+// Self-test of the failure path the convolution kernels share: a wait on a barrier that nobody will
+// ever complete runs out of its poll budget, the block reports through the status word exactly as
+// the kernels do, and returns normally.
+__global__ void k_wait_expiry(int* status, uint32_t polls)
+{
+    __shared__ uint64_t bar;
+    const uint32_t b = nmk::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        nmk::mbar_init(b, 1);
+        nmk::mbar_fence_init();
+    }
+    __syncthreads();
+    const bool ok = nmk::mbar_wait_polls(b, 0, polls);
+    if (!__syncthreads_and(ok ? 1 : 0) && threadIdx.x == 0) {
+        atomicExch(status + 0, static_cast<int>(NM_ERR_TIMEOUT));
+        atomicExch(status + 1, 99);   // where: the self-test
+        atomicExch(status + 2, static_cast<int>(blockIdx.x));
+    }
+}
+
 }  // namespace
+
+extern "C" nm_status_t nm_selftest_wait_expiry(const nm_weights_t* w, void* cuda_stream)
+{
+    if (!w || w->magic != NM_MAGIC) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_selftest_wait_expiry: bad weights handle");
+    k_wait_expiry<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(w->status, 2000u);
+    nmhost::count_launch(1);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_selftest_wait_expiry launch: %s", cudaGetErrorString(e));
+    return NM_OK;
+}
 
 extern "C" nm_status_t nm_maxpool2d(const float* x, int batch, int h, int w, int c, int kh, int kw, int stride_h,
                                     int stride_w, int pad_h, int pad_w, float* y, void* cuda_stream)

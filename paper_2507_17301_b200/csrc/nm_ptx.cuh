@@ -98,6 +98,14 @@ struct RingPos {
     }
 };
 
+// The same wait with an explicit poll budget (self-test of the expiry path).
+__device__ __forceinline__ bool mbar_wait_polls(uint32_t bar, uint32_t parity, uint32_t polls)
+{
+    for (uint32_t i = 0; i < polls; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
 // Wait that is usually already satisfied (a stage of a full pipeline): one non-blocking test first
 // (it returns in less than half the time of the blocking form when the phase is complete), then
 // the bounded blocking wait.  The test is made once, not in a loop: many lanes spinning on

@@ -53,6 +53,8 @@ def _load():
     lib.nm_weights_export.argtypes = [vp, vp, vp, vp]
     lib.nm_weights_import.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, ctypes.POINTER(vp)]
     lib.nm_weights_check.argtypes = [vp, vp]
+    lib.nm_selftest_wait_expiry.argtypes = [vp, vp]
+    lib.nm_selftest_wait_expiry.restype = ctypes.c_int
     lib.nm_maxpool2d.argtypes = [vp] + [i] * 10 + [vp, vp]
     lib.nm_maxpool2d.restype = ctypes.c_int
     lib.nm_weights_retained_l1.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
@@ -83,7 +85,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_maxpool2d", "nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_selftest_wait_expiry", "nm_maxpool2d", "nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -228,6 +230,11 @@ def nm_weights_retained_l1(w: Weights):
     kept, total = ctypes.c_double(), ctypes.c_double()
     _check(_lib.nm_weights_retained_l1(w.handle, ctypes.byref(kept), ctypes.byref(total)))
     return float(kept.value), float(total.value)
+
+
+def nm_selftest_wait_expiry(w: Weights):
+    """Makes a bounded device-side wait run out on purpose; the next ``nm_weights_check`` raises NM_ERR_TIMEOUT."""
+    _check(_lib.nm_selftest_wait_expiry(w.handle, _stream()))
 
 
 def nm_weights_check(w: Weights):

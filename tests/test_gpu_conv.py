@@ -321,6 +321,25 @@ def test_argument_errors(nm):
     assert torch.isfinite(y).all()
 
 
+def test_expired_wait_is_reported_and_the_context_survives(nm):
+    """A device-side wait that runs out (on a barrier nothing completes) ends its kernel normally, is
+    reported once through the status word, and leaves the handle and the context usable."""
+    s = inputs.config_tiny()
+    w, x, b = tensors_for(s)
+    _, _, yr = oracle_layer(s, w, x, b)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    nm.nm_weights_check(hnd)                                   # clean to begin with
+    nm.nm_selftest_wait_expiry(hnd)
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_weights_check(hnd)
+    assert e.value.status == nm.NM_ERR_TIMEOUT
+    nm.nm_weights_check(hnd)                                   # reported once, then cleared
+    y = nm.nm_conv2d(hnd, x.cuda(), s.kh, s.kw, s.stride, s.pad, s.dil, b.cuda(), s.relu)
+    nm.nm_weights_check(hnd)
+    torch.cuda.synchronize()
+    assert_conv_close(y.cpu().numpy(), yr)
+
+
 def test_host_buffer_entry_point(nm):
     s = inputs.config_tiny()
     w, x, b = tensors_for(s)
