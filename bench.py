@@ -39,9 +39,10 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 TF32_OVER_BF16 = 1.1 / 2.25   # nominal dense tensor peaks: 1.1 PFLOP/s TF32, 2.25 PFLOP/s bf16
 KERNEL_OF_VARIANT = {1: "k_conv_gather", 2: "k_conv_slab", 3: "k_conv_stream", 4: "k_conv_expand", 5: "k_conv_rowrun",
-                     6: "k_conv_window"}
+                     6: "k_conv_window", 7: "k_conv_pair"}
 KERNEL_SOURCE = {"k_conv_gather": "nm_conv_gather.cu", "k_conv_slab": "nm_conv_slab.cu", "k_conv_stream": "nm_conv_stream.cu",
-                 "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu", "k_conv_window": "nm_conv_window.cu"}
+                 "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu", "k_conv_window": "nm_conv_window.cu",
+                 "k_conv_pair": "nm_conv_pair.cu"}
 
 
 def peaks():
@@ -307,6 +308,7 @@ def main():
     ap.add_argument("--bn", type=int, default=0, help="with --variant: output channels per CTA")
     ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
     ap.add_argument("--split", type=int, default=0, help="with --variant: the plan's split field")
+    ap.add_argument("--kblk", type=int, default=0, help="with --variant: 32-column blocks per pipeline stage")
     ap.add_argument("--depth", type=int, default=50, choices=[18, 34, 50, 101, 152], help="ResNet depth of the conv stack")
     ap.add_argument("--nm", default="2:4", help="N:M pattern of the pruned layers, e.g. 1:4 or 2:8")
     ap.add_argument("--tile", type=int, default=64, help="pruning tile width T")
@@ -355,12 +357,14 @@ def main():
         if loaded is not None and s.name in loaded:
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.stages, plan.split = (loaded[s.name][k] for k in ("variant", "bn", "stages", "split"))
+            plan.kblk = loaded[s.name].get("kblk", 0)
             nm.nm_weights_reserve(hnd, nm.nm_plan_scratch_bytes(hnd, x.shape, s.stride, s.pad, s.dil, plan))
         elif args.variant is None:
             plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
         else:
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.stages, plan.split = args.variant, args.bn, args.stages, args.split
+            plan.kblk = args.kblk
         state.append((s, hnd, x, bias, y, plan))
 
     if args.save_plans and rank == 0:

@@ -75,14 +75,21 @@ typedef struct nm_weights nm_weights_t;
  *                input patch per 32-channel block in shared memory, every tap a shifted view of it
  *                (needs stride 1, c_in % 32 == 0, c_out % 32 == 0, w + 2 * pad_w <= 256; expanded
  *                weights as in variant 4).
+ *            7 = pair kernel: variant 4 run by clusters of two CTAs (tcgen05 cta_group::2), each SM
+ *                staging its own 128 pixels and half of the weight rows of a 256 x bn MMA, which
+ *                halves the shared-memory traffic per FLOP on reduction-heavy layers (needs the
+ *                conditions of variant 4, bn 128 or 256, c_out % bn == 0).
  *   bn       output channels per CTA / work item (variants 2, 3: a multiple of tile_t; variant 4: a
- *            multiple of 32 up to 256; variant 6 likewise), 0 = default
+ *            multiple of 32 up to 256; variant 6 likewise; variant 7: 128 or 256), 0 = default
  *   stages   depth of the shared-memory ring, 0 = default
  *   split    variant 2: 1 = cp.async producer, 2 = direct-store epilogue; variant 4: 0 = keep a CTA's weight
  *            slice resident in shared memory when it fits, 1 = stream the weights with the activations,
  *            2-8 = number of CTAs the reduction axis is split over ( partial sums go through scratch memory that nm_autotune
  *            reserves on the handle, so such a plan works only on a handle nm_autotune has seen with a
  *            layer at least as large); variant 6: M-tiles per work item (1-4); otherwise 0
+ *   kblk     variants 4 and 7: 32-column blocks of the reduction axis per pipeline stage, 1 or 2 (0 = 1);
+ *            two blocks halve the barrier round trips per MMA, which pays where the MMAs are short
+ *            (few channels per work item) or the layer is small; K / 32 (per split) must be a multiple
  * A plan the layer does not admit gives NM_ERR_UNSUPPORTED.
  */
 typedef struct {
@@ -90,7 +97,8 @@ typedef struct {
     int bn;
     int stages;
     int split;
-    int reserved[12];
+    int kblk;
+    int reserved[11];
 } nm_plan_t;
 
 /* ---------------------------------------------------------------------------------------------
@@ -268,6 +276,11 @@ nm_status_t nm_maxpool2d(const float* x, int batch, int h, int w, int c, int kh,
  * several), writes the fastest to *best and its time to *best_ms (may be NULL).  x and y_scratch
  * are caller buffers of the sizes nm_conv2d expects; y_scratch is overwritten.  Synchronises the
  * stream.  A candidate that fails to launch is skipped; NM_ERR_UNSUPPORTED if none runs.
+ * Every timed launch starts with a cold L2: the call allocates a 288 MiB buffer for its own
+ * duration and overwrites it before each launch (if that allocation fails the launches run warm), so
+ * layers that would fit the cache are tuned for operands that come from HBM.  Candidates are tried
+ * most promising first and a later one replaces the best so far only if it is at least 1 % faster.
+ * This call allocates (the buffer above, and the split-K scratch described at nm_weights_reserve).
  * The environment variable NM_AUTOTUNE_VARIANTS (a list of variant digits such as "1,2,3") restricts the
  * search, e.g. to the kernels that skip the pruned columns.
  */

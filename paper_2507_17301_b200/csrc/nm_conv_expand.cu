@@ -45,7 +45,9 @@ struct ExpandCfg {
     int stage_bytes;
     int w_res;        // 1: this CTA's weight slice stays resident in shared memory (it is loaded once)
     int wres_bytes;   // bytes of the resident slice: all 32-column blocks of bn rows
-    int n_sub;        // 32-column blocks one work item reduces over: (K / 32) / ksplit
+    int n_sub;        // pipeline stages one work item reduces over: (K / 32) / ksplit / kblk
+    int kblk;         // 32-column blocks per stage (1 or 2): one barrier round trip then covers kblk * 4 MMAs
+    int sub_bytes;    // bytes of one 32-column block inside a stage: activations (+ streamed weights)
     int ksplit;       // K splits (1 = none): a work item covers one of them and stores raw partial sums
     int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
     int boxes;        // output staging boxes per epilogue warp: 2 for short reductions, 1 when the ring needs the room
@@ -99,13 +101,14 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         if (lane == 0) {
             int issued = 0;
             const int hw = p.ho * p.wo;
-            const uint32_t tx = SUB_BYTES + (cfg.w_res ? 0u : static_cast<uint32_t>(cfg.bn) * 128u);
+            const uint32_t tx = static_cast<uint32_t>(cfg.kblk) * (SUB_BYTES + (cfg.w_res ? 0u : static_cast<uint32_t>(cfg.bn) * 128u));
+            const int n_blk32 = n_sub * cfg.kblk;   // 32-column blocks per work item
             if (cfg.w_res) {
                 // the grid is a multiple of the slice count, so every work item of this CTA has the
                 // same channel slice: its weights are fetched once
                 const int slice = static_cast<int>(blockIdx.x % static_cast<uint32_t>(cfg.n_slices));
-                mbar_arrive_expect_tx(smem_u32(&s_wres), static_cast<uint32_t>(n_sub) * static_cast<uint32_t>(cfg.bn) * 128u);
-                for (int c = 0; c < n_sub; ++c)
+                mbar_arrive_expect_tx(smem_u32(&s_wres), static_cast<uint32_t>(n_blk32) * static_cast<uint32_t>(cfg.bn) * 128u);
+                for (int c = 0; c < n_blk32; ++c)
                     bulk_load_1d(wres + c * cfg.b_bytes, p.wx + (static_cast<size_t>(c) * p.c_out + slice * cfg.bn) * 32,
                                  static_cast<uint32_t>(cfg.bn) * 128u, smem_u32(&s_wres));
             }
@@ -122,7 +125,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
                 // first 32-column block of this item's share of the reduction axis
-                const int c0 = ks * n_sub;
+                const int c0 = ks * n_blk32;
                 const int tap0 = (c0 * 32) / p.c_in;
                 const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32 + static_cast<size_t>(c0) * w_step;
                 int ch = c0 * 32 - tap0 * p.c_in, tw = tap0 % p.kw;
@@ -130,18 +133,21 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 for (int c = 0; c < n_sub; ++c) {
                     if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
-                    const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
+                    uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     const uint32_t bar = smem_u32(&s_full[rp.s]);
                     mbar_arrive_expect_tx(bar, tx);
-                    tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>(off_w),
-                                       static_cast<uint16_t>(off_h));
-                    if (!cfg.w_res) bulk_load_1d(a_smem + SUB_BYTES, wsrc, w_bytes, bar);
-                    wsrc += w_step;
-                    ch += 32;
-                    if (ch >= p.c_in) {
-                        ch = 0;
-                        off_w += p.dil_w;
-                        if (++tw == p.kw) { tw = 0; off_w = 0; off_h += p.dil_h; }
+                    for (int j = 0; j < cfg.kblk; ++j) {
+                        tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>(off_w),
+                                           static_cast<uint16_t>(off_h));
+                        if (!cfg.w_res) bulk_load_1d(a_smem + SUB_BYTES, wsrc, w_bytes, bar);
+                        a_smem += cfg.sub_bytes;
+                        wsrc += w_step;
+                        ch += 32;
+                        if (ch >= p.c_in) {
+                            ch = 0;
+                            off_w += p.dil_w;
+                            if (++tw == p.kw) { tw = 0; off_w = 0; off_h += p.dil_h; }
+                        }
                     }
                     rp.advance(NS);
                     ++issued;
@@ -176,11 +182,16 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     if (!mbar_wait_lone(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     tc_fence_after();
                     const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
-                    const uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
-                    const uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
+                    uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
+                    uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * cfg.kblk * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
+                    const uint32_t b_step = static_cast<uint32_t>(cfg.w_res ? cfg.b_bytes : cfg.sub_bytes) >> 4;
+                    for (int j = 0; j < cfg.kblk; ++j) {
 #pragma unroll
-                    for (int kq = 0; kq < 4; ++kq)
-                        umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > 0 || kq > 0) ? 1u : 0u);
+                        for (int kq = 0; kq < 4; ++kq)
+                            umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > 0 || j > 0 || kq > 0) ? 1u : 0u);
+                        adesc += static_cast<uint32_t>(cfg.sub_bytes) >> 4;   // next 32-column block (start address field, 16-byte units)
+                        bdesc += b_step;
+                    }
                     umma_commit(smem_u32(&s_free[rp.s]));
                     rp.advance(NS);
                 }
@@ -347,23 +358,28 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     const int splits = plan && plan->split > 1 ? plan->split : 1;
     if (splits > 8 || (p.k / 32) % splits != 0) return false;
     cfg->ksplit = splits;
-    cfg->n_sub = (p.k / 32) / splits;
+    const int blk32 = (p.k / 32) / splits;   // 32-column blocks per work item
+    const int kblk = plan && plan->kblk > 0 ? plan->kblk : 1;
+    if (kblk > 2 || blk32 % kblk != 0) return false;
+    cfg->kblk = kblk;
+    cfg->n_sub = blk32 / kblk;
     cfg->p_pad = static_cast<int>(((p.pixels + BM - 1) / BM) * BM);
     if (splits > 1 && (!p.splitk || p.splitk_bytes < static_cast<size_t>(splits) * cfg->p_pad * p.c_out * sizeof(float) ||
                        static_cast<long long>(splits) * cfg->p_pad >= (1ll << 31)))
         return false;   // the partial-sum scratch is reserved by nm_autotune
-    cfg->boxes = cfg->n_sub <= 8 ? 2 : 1;   // long reductions: the epilogue is rare, the ring needs the bytes
+    cfg->boxes = blk32 <= 8 ? 2 : 1;   // long reductions: the epilogue is rare, the ring needs the bytes
     // A weight slice that fits stays resident (plan.split == 1 asks for streaming instead): the ring
     // then holds activations only and is deeper.  Needs one fixed slice per CTA, i.e. a grid that is a
     // multiple of the slice count.
     cfg->wres_bytes = 0;
     cfg->w_res = 0;
-    if (splits == 1 && !(plan && plan->split == 1) && cfg->n_sub * cfg->b_bytes <= WRES_MAX && cfg->n_slices <= sm_count()) {
+    if (splits == 1 && !(plan && plan->split == 1) && blk32 * cfg->b_bytes <= WRES_MAX && cfg->n_slices <= sm_count()) {
         cfg->w_res = 1;
-        cfg->wres_bytes = cfg->n_sub * cfg->b_bytes;
+        cfg->wres_bytes = blk32 * cfg->b_bytes;
         if (cfg->wres_bytes > 64 * 1024) cfg->boxes = 1;   // a large slice: give the output staging's room to the ring
     }
-    cfg->stage_bytes = SUB_BYTES + (cfg->w_res ? 0 : cfg->b_bytes);
+    cfg->sub_bytes = SUB_BYTES + (cfg->w_res ? 0 : cfg->b_bytes);
+    cfg->stage_bytes = kblk * cfg->sub_bytes;
     const int budget = 227 * 1024 - 1024 - 8 * cfg->boxes * BOX_BYTES - 1024 - cfg->wres_bytes;
     int stages = plan && plan->stages > 0 ? plan->stages : NSTAGE_MAX;
     if (stages > NSTAGE_MAX) return false;

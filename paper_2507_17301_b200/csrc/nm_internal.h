@@ -127,6 +127,10 @@ nm_status_t launch_conv_rowrun(const ConvParams& p, const nm_plan_t* plan, cudaS
 bool window_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_window(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 
+// nm_conv_pair.cu — variant 7
+bool pair_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_pair(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
 // nm_conv_stream.cu — variant 3
 bool stream_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_stream(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);

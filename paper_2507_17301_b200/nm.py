@@ -32,10 +32,11 @@ class NmError(RuntimeError):
 
 class nm_plan_t(ctypes.Structure):
     _fields_ = [("variant", ctypes.c_int), ("bn", ctypes.c_int), ("stages", ctypes.c_int),
-                ("split", ctypes.c_int), ("reserved", ctypes.c_int * 12)]
+                ("split", ctypes.c_int), ("kblk", ctypes.c_int), ("reserved", ctypes.c_int * 11)]
 
     def as_dict(self):
-        return {"variant": self.variant, "bn": self.bn, "stages": self.stages, "split": self.split}
+        return {"variant": self.variant, "bn": self.bn, "stages": self.stages, "split": self.split,
+                "kblk": self.kblk}
 
 
 def _load():

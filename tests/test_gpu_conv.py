@@ -31,9 +31,10 @@ def _plans(nm, s):
         out.append(p)
     # expanded-operand kernel: default width, 32 and 256 channels per work item, two-stage ring, and
     # (split = 1) weights streamed per stage instead of kept resident
-    for bn, stages, split in ((0, 0, 0), (32, 0, 0), (256, 0, 0), (0, 2, 0), (0, 0, 1), (64, 0, 1)):
+    for bn, stages, split, kblk in ((0, 0, 0, 0), (32, 0, 0, 0), (256, 0, 0, 0), (0, 2, 0, 0), (0, 0, 1, 0), (64, 0, 1, 0),
+                                    (0, 0, 0, 2), (128, 2, 1, 2), (256, 0, 1, 2)):   # kblk = 2: two 32-column blocks per stage
         p = nm.nm_plan_t()
-        p.variant, p.bn, p.stages, p.split = 4, bn, stages, split
+        p.variant, p.bn, p.stages, p.split, p.kblk = 4, bn, stages, split, kblk
         out.append(p)
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
@@ -42,6 +43,11 @@ def _plans(nm, s):
     for bn, mt, stages in ((0, 0, 0), (64, 1, 0), (0, 2, 0), (32, 1, 3), (64, 3, 0), (32, 4, 0), (128, 4, 0)):
         p = nm.nm_plan_t()
         p.variant, p.bn, p.split, p.stages = 6, bn, mt, stages
+        out.append(p)
+    # pair kernel (clusters of two CTAs): default, both widths, a two-stage ring
+    for bn, stages, kblk in ((0, 0, 0), (128, 0, 1), (256, 0, 1), (128, 2, 2)):
+        p = nm.nm_plan_t()
+        p.variant, p.bn, p.stages, p.kblk = 7, bn, stages, kblk
         out.append(p)
     return out
 
@@ -176,6 +182,26 @@ def test_window_shapes_integer_exact(nm, s):
     _run(nm, s, integer=True, need_variant=[6])
 
 
+# pair kernel (variant 7): clusters of two CTAs share one 256-pixel x bn MMA
+PAIR = [
+    ConvShape("pair_one", 1, 16, 16, 128, 256, 3, 3, 1, 1, 1, 2, 4, 64),              # 2 pixel blocks: one pair, one item
+    ConvShape("pair_odd_blocks", 2, 13, 13, 128, 256, 3, 3, 1, 1, 1, 2, 4, 64),       # 338 pixels: 3 blocks, the 4th is empty
+    ConvShape("pair_1x1_long_k", 2, 14, 14, 1024, 128, 1, 1, 1, 0, 1, 2, 4, 64),      # 32 stages: the ring wraps
+    ConvShape("pair_stride2", 2, 29, 29, 64, 128, 3, 3, 2, 1, 1, 1, 4, 32),
+    ConvShape("pair_many_items", 8, 56, 56, 32, 256, 3, 3, 1, 1, 1, 2, 4, 64),        # 98 block pairs x 1-2 slices: several items per pair
+]
+
+
+@pytest.mark.parametrize("s", PAIR, ids=lambda s: s.name)
+def test_pair_shapes(nm, s):
+    _run(nm, s, need_variant=[4, 7])
+
+
+@pytest.mark.parametrize("s", PAIR[:4], ids=lambda s: s.name)
+def test_pair_shapes_integer_exact(nm, s):
+    _run(nm, s, integer=True, need_variant=[7])
+
+
 @pytest.mark.parametrize("s", MEDIUM, ids=lambda s: s.name)
 def test_medium_shapes(nm, s):
     # the stream kernel takes tiles that are multiples of 16 channels and its seven N:M patterns
@@ -246,6 +272,7 @@ def test_split_k_plans(nm, integer):
         for bn in (32, 64):
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.split = 4, bn, splits
+            plan.kblk = 2 if bn == 64 else 0                  # K / 32 / splits = 36, 24, 18: two blocks per stage fit
             for _ in range(2):                                # twice: the scratch is reused
                 y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
             nm.nm_weights_check(hnd)
