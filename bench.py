@@ -365,6 +365,7 @@ def main():
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.stages, plan.split = args.variant, args.bn, args.stages, args.split
             plan.kblk = args.kblk
+            nm.nm_weights_reserve(hnd, nm.nm_plan_scratch_bytes(hnd, x.shape, s.stride, s.pad, s.dil, plan))
         state.append((s, hnd, x, bias, y, plan))
 
     if args.save_plans and rank == 0:

@@ -86,7 +86,11 @@ typedef struct nm_weights nm_weights_t;
  *            slice resident in shared memory when it fits, 1 = stream the weights with the activations,
  *            2-8 = number of CTAs the reduction axis is split over ( partial sums go through scratch memory that nm_autotune
  *            reserves on the handle, so such a plan works only on a handle nm_autotune has seen with a
- *            layer at least as large); variant 6: M-tiles per work item (1-4); otherwise 0
+ *            layer at least as large), -1 = balanced: the (work item, stage) pairs of the layer are cut into
+ *            one equal contiguous range per SM, an item shared by several CTAs is completed by the CTA
+ *            that holds its first stage from the others' partial sums (per-SM slots in the same
+ *            scratch; for layers with too few work items to fill every SM evenly);
+ *            variant 6: M-tiles per work item (1-4); otherwise 0
  *   kblk     variants 4 and 7: 32-column blocks of the reduction axis per pipeline stage, 1 or 2 (0 = 1);
  *            two blocks halve the barrier round trips per MMA, which pays where the MMAs are short
  *            (few channels per work item) or the layer is small; K / 32 (per split) must be a multiple

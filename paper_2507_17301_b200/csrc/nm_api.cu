@@ -185,6 +185,13 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
         a.variant = 7; a.bn = bn; a.stages = 0; a.split = 0;
         if (nmhost::pair_plan_ok(p, &a)) out.push_back(a);
     }
+    for (int bn : {256, 128}) {             // ... with (item, stage) ranges balanced over the SMs (needs the handle's scratch)
+        for (int kblk : {1, 2}) {
+            a.variant = 4; a.bn = bn; a.stages = 0; a.split = -1; a.kblk = kblk;
+            if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);
+        }
+    }
+    a.kblk = 0;
     for (int splits : {2, 3, 4}) {          // ... with the reduction axis split (needs the handle's scratch)
         for (int bn : {128, 256}) {
             for (int kblk : {1, 2}) {
@@ -327,6 +334,7 @@ nm_status_t nm_plan_scratch_bytes(const nm_weights_t* w, int batch, int h, int w
                                 dil_h, dil_w, nullptr, 0, dummy, &p);
     if (s != NM_OK) return s;
     if (plan && plan->variant == 4 && plan->split > 1) *bytes = nmhost::expand_splitk_bytes(p, plan->split);
+    if (plan && plan->variant == 4 && plan->split == -1) *bytes = nmhost::expand_balanced_bytes(plan->bn > 0 ? plan->bn : 256);
     return NM_OK;
 }
 
@@ -341,6 +349,13 @@ nm_status_t nm_weights_reserve(nm_weights_t* w, size_t bytes)
     if (cudaMalloc(&w->splitk, bytes) != cudaSuccess) {
         (void)cudaGetLastError();
         return nmhost::fail(NM_ERR_ALLOC, "nm_weights_reserve: cannot allocate %zu bytes", bytes);
+    }
+    // balanced plans keep flag words in the scratch: they start cleared
+    if (cudaMemset(w->splitk, 0, bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaFree(w->splitk);
+        w->splitk = nullptr;
+        return nmhost::fail(NM_ERR_CUDA, "nm_weights_reserve: cannot clear the scratch");
     }
     w->splitk_bytes = bytes;
     return NM_OK;
@@ -443,7 +458,10 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         const long long pix_blocks = (p.pixels + 127) / 128;
         const bool few_items = pix_blocks * ((p.c_out + 255) / 256) < n_sm && p.k / 32 >= 32;
-        const size_t need = few_items && p.wx ? nmhost::expand_splitk_bytes(p, 4) : 0;
+        size_t need = few_items && p.wx ? nmhost::expand_splitk_bytes(p, 4) : 0;
+        // ... and layers with fewer than three rounds of work items with (item, stage) ranges balanced over the SMs
+        const bool uneven = pix_blocks * ((p.c_out + 255) / 256) < 3ll * n_sm;
+        if (uneven && p.wx && nmhost::expand_balanced_bytes(256) > need) need = nmhost::expand_balanced_bytes(256);
         if (need > hw->splitk_bytes) (void)nm_weights_reserve(hw, need);   // no scratch: the split plans are simply not candidates
         p.splitk = hw->splitk;
         p.splitk_bytes = hw->splitk_bytes;

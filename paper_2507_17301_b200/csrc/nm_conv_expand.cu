@@ -22,6 +22,18 @@
 //                         overlaps the next work item's main loop
 // Work items (128 pixels x BN channels) are walked in a static persistent schedule; every wait is
 // bounded and reports through the handle's status word.
+//
+// Balanced mode (plan.split = -1), for layers with fewer work items than would keep every SM busy:
+// the (item, stage) pairs of the whole layer are laid end to end and cut into one contiguous,
+// equally long range per CTA, so an item may be shared by two or more CTAs.  A CTA whose range
+// begins inside an item handles that part FIRST, stores the raw partial accumulator to its own
+// slot of the handle's scratch and raises a per-warp flag; the CTA whose range holds the item's
+// first stage handles it LAST, waits (bounded) for the flags of the others, adds their partial sums
+// to its accumulator and runs the normal epilogue.  Ranges are handed out from the end of the
+// layer to CTA 0 upwards, so a CTA only ever waits for CTAs with a lower index, whose first action
+// is the store it waits for.
+#include <atomic>
+
 #include "nm_internal.h"
 #include "nm_ptx.cuh"
 #include "nm_tmap.cuh"
@@ -51,11 +63,77 @@ struct ExpandCfg {
     int ksplit;       // K splits (1 = none): a work item covers one of them and stores raw partial sums
     int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
     int boxes;        // output staging boxes per epilogue warp: 2 for short reductions, 1 when the ring needs the room
+    int balanced;     // 1: contiguous (item, stage) ranges per CTA, partial sums through per-CTA scratch slots
+    uint32_t epoch;   // balanced mode: value the flags of this launch carry
     long long n_work;
 };
 
 __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
 
+// One piece of work of a CTA: stages [sb, se) of work item `work`.
+struct Seg {
+    uint32_t work;
+    int sb, se;
+};
+// Walks a CTA's pieces: whole items `first, first + stride, ...` in the static schedule, or the
+// contiguous range of (item, stage) units of balanced mode.
+template <bool BAL>
+struct SegIter {
+    uint32_t cur, end, stride;
+    int stages;
+    __device__ __forceinline__ bool next(Seg& g)
+    {
+        if (cur >= end) return false;
+        if (!BAL) {
+            g.work = cur; g.sb = 0; g.se = stages;
+            cur += stride;
+            return true;
+        }
+        g.work = cur / static_cast<uint32_t>(stages);
+        g.sb = static_cast<int>(cur - g.work * static_cast<uint32_t>(stages));
+        const uint32_t left = end - cur, room = static_cast<uint32_t>(stages - g.sb);
+        const int len = static_cast<int>(left < room ? left : room);
+        g.se = g.sb + len;
+        cur += static_cast<uint32_t>(len);
+        return true;
+    }
+};
+// First (item, stage) unit of the range at position j of `n` equal ranges over `units`.
+__device__ __forceinline__ uint32_t range_begin(uint32_t j, uint32_t n, uint32_t units)
+{
+    return static_cast<uint32_t>(static_cast<unsigned long long>(j) * units / n);
+}
+template <bool BAL>
+__device__ __forceinline__ SegIter<BAL> make_iter(const ExpandCfg& cfg)
+{
+    SegIter<BAL> it;
+    it.stages = cfg.n_sub;
+    if (!BAL) {
+        it.cur = blockIdx.x; it.end = static_cast<uint32_t>(cfg.n_work); it.stride = gridDim.x;
+    } else {
+        // ranges are handed out from the end of the layer: CTA b takes position gridDim.x - 1 - b
+        const uint32_t units = static_cast<uint32_t>(cfg.n_work) * static_cast<uint32_t>(cfg.n_sub);
+        const uint32_t j = gridDim.x - 1u - blockIdx.x;
+        it.cur = range_begin(j, gridDim.x, units);
+        it.end = range_begin(j + 1u, gridDim.x, units);
+        it.stride = 0;
+    }
+    return it;
+}
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* ptr)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(uint32_t* ptr, uint32_t v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+
+// KBLK: 32-column blocks per pipeline stage; BAL: balanced mode.  Compile-time, so that the lone producer and
+// issuer threads of the common configuration (1, false) run exactly the instructions they need.
+template <int KBLK, bool BAL>
 __global__ void __launch_bounds__(THREADS, 1)
 k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ CUtensorMap tm_x,
               const __grid_constant__ CUtensorMap tm_y)
@@ -66,7 +144,6 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t n_work = static_cast<uint32_t>(cfg.n_work);   // below 2^31: per-item arithmetic stays 32-bit
     const int NS = cfg.stages, n_sub = cfg.n_sub;
     const uint32_t wres = (smem_u32(smem_raw) + 1023u) & ~1023u;   // resident weight slice (may be empty)
     const uint32_t ring = wres + cfg.wres_bytes;
@@ -101,8 +178,8 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         if (lane == 0) {
             int issued = 0;
             const int hw = p.ho * p.wo;
-            const uint32_t tx = static_cast<uint32_t>(cfg.kblk) * (SUB_BYTES + (cfg.w_res ? 0u : static_cast<uint32_t>(cfg.bn) * 128u));
-            const int n_blk32 = n_sub * cfg.kblk;   // 32-column blocks per work item
+            const uint32_t tx = static_cast<uint32_t>(KBLK) * (SUB_BYTES + (cfg.w_res ? 0u : static_cast<uint32_t>(cfg.bn) * 128u));
+            const int n_blk32 = n_sub * KBLK;   // 32-column blocks per work item
             if (cfg.w_res) {
                 // the grid is a multiple of the slice count, so every work item of this CTA has the
                 // same channel slice: its weights are fetched once
@@ -115,7 +192,10 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
             const size_t w_step = static_cast<size_t>(p.c_out) * 32;   // floats between two 32-column blocks
             RingPos rp;
-            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
+            SegIter<BAL> it = make_iter<BAL>(cfg);
+            Seg seg;
+            while (!aborted(abort_flag) && it.next(seg)) {
+                const uint32_t work = seg.work;
                 const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
                 const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
                 const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
@@ -125,18 +205,19 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
                 // first 32-column block of this item's share of the reduction axis
-                const int c0 = ks * n_blk32;
+                const int c0 = ks * n_blk32 + seg.sb * KBLK;
                 const int tap0 = (c0 * 32) / p.c_in;
                 const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32 + static_cast<size_t>(c0) * w_step;
                 int ch = c0 * 32 - tap0 * p.c_in, tw = tap0 % p.kw;
                 int off_w = tw * p.dil_w, off_h = (tap0 / p.kw) * p.dil_h;
-                for (int c = 0; c < n_sub; ++c) {
+                for (int c = seg.sb; c < seg.se; ++c) {
                     if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
                     uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     const uint32_t bar = smem_u32(&s_full[rp.s]);
                     mbar_arrive_expect_tx(bar, tx);
-                    for (int j = 0; j < cfg.kblk; ++j) {
+#pragma unroll
+                    for (int j = 0; j < KBLK; ++j) {
                         tma_load_im2col_4d(a_smem, &tm_x, bar, ch, w0, h0, n0, static_cast<uint16_t>(off_w),
                                            static_cast<uint16_t>(off_h));
                         if (!cfg.w_res) bulk_load_1d(a_smem + SUB_BYTES, wsrc, w_bytes, bar);
@@ -171,26 +252,31 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             RingPos rp;
             uint32_t ab = 0, acc_par = 0;   // accumulator buffer of this item, parity of its current use
             bool acc_wrapped = false;
-            for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
+            SegIter<BAL> it = make_iter<BAL>(cfg);
+            Seg seg;
+            while (!aborted(abort_flag) && it.next(seg)) {
                 if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
                     *abort_flag = 5;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
-                for (int c = 0; c < n_sub; ++c) {
+                for (int c = seg.sb; c < seg.se; ++c) {
                     if (!mbar_wait_lone(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     tc_fence_after();
                     const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
-                    uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * cfg.kblk * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
-                    const uint32_t b_step = static_cast<uint32_t>(cfg.w_res ? cfg.b_bytes : cfg.sub_bytes) >> 4;
-                    for (int j = 0; j < cfg.kblk; ++j) {
+                    uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * KBLK * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
+                    const uint32_t b_step = KBLK > 1 ? static_cast<uint32_t>(cfg.w_res ? cfg.b_bytes : cfg.sub_bytes) >> 4 : 0u;
+#pragma unroll
+                    for (int j = 0; j < KBLK; ++j) {
 #pragma unroll
                         for (int kq = 0; kq < 4; ++kq)
-                            umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > 0 || j > 0 || kq > 0) ? 1u : 0u);
-                        adesc += static_cast<uint32_t>(cfg.sub_bytes) >> 4;   // next 32-column block (start address field, 16-byte units)
-                        bdesc += b_step;
+                            umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > seg.sb || j > 0 || kq > 0) ? 1u : 0u);
+                        if (j + 1 < KBLK) {
+                            adesc += static_cast<uint32_t>(cfg.sub_bytes) >> 4;   // next 32-column block (start address field, 16-byte units)
+                            bdesc += b_step;
+                        }
                     }
                     umma_commit(smem_u32(&s_free[rp.s]));
                     rp.advance(NS);
@@ -211,7 +297,17 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t nb = 0, ti = 0;
-        for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
+        // balanced mode: this CTA's partial-sum slot (128 rows x bn) and its warps' flags, in the handle's scratch
+        const uint32_t units = static_cast<uint32_t>(cfg.n_work) * static_cast<uint32_t>(cfg.n_sub);
+        const size_t slot_floats = static_cast<size_t>(BM) * cfg.bn;
+        uint32_t* const flags = reinterpret_cast<uint32_t*>(p.splitk + slot_floats * gridDim.x);
+        const int my_row = q * 32 + lane;
+        SegIter<BAL> it = make_iter<BAL>(cfg);
+        Seg seg;
+        for (; it.next(seg); ++ti) {
+            const uint32_t work = seg.work;
+            const bool publish = BAL && seg.sb > 0;                   // a later part of an item: store raw sums
+            const bool finish = BAL && seg.sb == 0 && seg.se < n_sub;  // the first part: add the others' sums
             const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
             const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
             const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
@@ -220,7 +316,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             // the shortcut input does not depend on the accumulator: its first box is requested before the
             // wait for the main loop, every later box while the one before it is being stored
             const long long box_pix = static_cast<long long>(pix0) + q * 32;
-            const bool res_pass = p.residual != nullptr && box_pix < p.pixels;
+            const bool res_pass = p.residual != nullptr && box_pix < p.pixels && !publish;
             const int res_rows = p.pixels - box_pix < 32 ? static_cast<int>(p.pixels - box_pix) : 32;
             const float* res_base = res_pass ? p.residual + box_pix * p.c_out + slice * cfg.bn : nullptr;
             float4 rv[8];
@@ -230,6 +326,23 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
             const int o0 = slice * cfg.bn;
+            // positions (of the equal ranges) that hold the rest of this item: first_pos + 1 .. last_pos
+            uint32_t first_pos = 0, last_pos = 0;
+            if (finish) {
+                first_pos = gridDim.x - 1u - blockIdx.x;
+                const uint32_t u_last = (work + 1u) * static_cast<uint32_t>(n_sub) - 1u;
+                last_pos = static_cast<uint32_t>(static_cast<unsigned long long>(u_last) * gridDim.x / units);
+                while (last_pos + 1u < gridDim.x && range_begin(last_pos + 1u, gridDim.x, units) <= u_last) ++last_pos;
+                while (last_pos > first_pos && range_begin(last_pos, gridDim.x, units) > u_last) --last_pos;
+                // each of this warp's counterparts has stored its rows and raised its flag (bounded wait)
+                for (uint32_t pos = first_pos + 1u; pos <= last_pos; ++pos) {
+                    const uint32_t* f = flags + (gridDim.x - 1u - pos) * 8u + (warp - 4);
+                    bool seen = false;
+                    for (uint32_t poll = 0; poll < kWaitPolls && !seen; ++poll) seen = ld_acquire_gpu(f) == cfg.epoch;
+                    if (!seen) *abort_flag = 10;
+                }
+                if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
+            }
             for (int blk = half; blk < n_blk; blk += 2, ++nb) {
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_addr + ab * cfg.bn + blk * 32, v);
@@ -238,6 +351,35 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+                }
+                if (publish) {
+                    // raw partial sums of this thread's row; the slot is laid out [channel quad][row], so the 32
+                    // lanes of a warp (32 consecutive rows) write 512 contiguous bytes per instruction
+                    float4* dst = reinterpret_cast<float4*>(p.splitk + slot_floats * blockIdx.x) +
+                                  static_cast<size_t>(blk) * 8 * BM + my_row;
+#pragma unroll
+                    for (int qq = 0; qq < 8; ++qq)
+                        __stcg(dst + qq * BM, make_float4(__uint_as_float(v[qq * 4 + 0]), __uint_as_float(v[qq * 4 + 1]),
+                                                     __uint_as_float(v[qq * 4 + 2]), __uint_as_float(v[qq * 4 + 3])));
+                    --nb;   // no staging box used
+                    continue;
+                }
+                if (finish) {
+                    for (uint32_t pos = first_pos + 1u; pos <= last_pos; ++pos) {
+                        const float4* src = reinterpret_cast<const float4*>(p.splitk + slot_floats * (gridDim.x - 1u - pos)) +
+                                            static_cast<size_t>(blk) * 8 * BM + my_row;
+                        float4 t4[8];
+#pragma unroll
+                        for (int qq = 0; qq < 8; ++qq) t4[qq] = __ldcg(src + qq * BM);
+#pragma unroll
+                        for (int qq = 0; qq < 8; ++qq) {
+                            const float4 t = t4[qq];
+                            v[qq * 4 + 0] = __float_as_uint(__uint_as_float(v[qq * 4 + 0]) + t.x);
+                            v[qq * 4 + 1] = __float_as_uint(__uint_as_float(v[qq * 4 + 1]) + t.y);
+                            v[qq * 4 + 2] = __float_as_uint(__uint_as_float(v[qq * 4 + 2]) + t.z);
+                            v[qq * 4 + 3] = __float_as_uint(__uint_as_float(v[qq * 4 + 3]) + t.w);
+                        }
+                    }
                 }
                 const uint32_t box = my_staging + (nb & box_toggle) * BOX_BYTES;
                 if (lane == 0) {
@@ -282,6 +424,12 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             if (n_blk == 1 && half == 1) {
                 // a single channel block: the second warp of the quadrant only releases the buffer
                 if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+            }
+            if (publish) {
+                // every lane's stores are ordered before the flag the reading warp acquires
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) st_release_gpu(flags + blockIdx.x * 8u + (warp - 4), cfg.epoch);
             }
         }
         if (lane == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads; the writes complete with the grid
@@ -356,6 +504,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     cfg->n_slices = p.c_out / bn;
     cfg->b_bytes = ((bn * 128 + 1023) / 1024) * 1024;
     const int splits = plan && plan->split > 1 ? plan->split : 1;
+    const bool balanced = plan && plan->split == -1;
     if (splits > 8 || (p.k / 32) % splits != 0) return false;
     cfg->ksplit = splits;
     const int blk32 = (p.k / 32) / splits;   // 32-column blocks per work item
@@ -373,7 +522,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     // multiple of the slice count.
     cfg->wres_bytes = 0;
     cfg->w_res = 0;
-    if (splits == 1 && !(plan && plan->split == 1) && blk32 * cfg->b_bytes <= WRES_MAX && cfg->n_slices <= sm_count()) {
+    if (splits == 1 && !balanced && !(plan && plan->split == 1) && blk32 * cfg->b_bytes <= WRES_MAX && cfg->n_slices <= sm_count()) {
         cfg->w_res = 1;
         cfg->wres_bytes = blk32 * cfg->b_bytes;
         if (cfg->wres_bytes > 64 * 1024) cfg->boxes = 1;   // a large slice: give the output staging's room to the ring
@@ -392,12 +541,27 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     cfg->stages = stages;
     cfg->n_work = ((p.pixels + BM - 1) / BM) * cfg->n_slices * splits;
     if (cfg->n_work >= (1ll << 31)) return false;
+    cfg->balanced = 0;
+    cfg->epoch = 0;
+    if (balanced) {
+        // one range per SM; needs at least one (item, stage) unit per CTA and the per-CTA slots + flags in the scratch
+        const long long units = cfg->n_work * cfg->n_sub;
+        if (units < sm_count() || units >= (1ll << 31)) return false;
+        if (!p.splitk || p.splitk_bytes < nmhost::expand_balanced_bytes(bn)) return false;
+        cfg->balanced = 1;
+    }
     return true;
 }
 
 }  // namespace
 
 namespace nmhost {
+
+size_t expand_balanced_bytes(int bn)
+{
+    // per SM: a slot of 128 rows x bn partial sums, and eight flag words (one per epilogue warp)
+    return static_cast<size_t>(sm_count()) * (static_cast<size_t>(BM) * bn * sizeof(float) + 8 * sizeof(uint32_t));
+}
 
 bool expand_plan_ok(const ConvParams& p, const nm_plan_t* plan)
 {
@@ -410,7 +574,7 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     ExpandCfg cfg;
     if (!make_cfg(p, plan, &cfg))
         return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the expanded-operand kernel does not take this layer / plan%s",
-                    plan && plan->split > 1 ? " (a split plan needs scratch: nm_weights_reserve)" : "");
+                    plan && (plan->split > 1 || plan->split == -1) ? " (a split or balanced plan needs scratch: nm_weights_reserve)" : "");
     // a split-K plan stores raw partial sums [split][pixel][channel] in the handle's scratch; bias and
     // activation are applied by the reduction pass
     ConvParams q = p;
@@ -427,11 +591,19 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     q.pixels = p.pixels;
     size_t smem = 1024 + cfg.wres_bytes + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 8 * cfg.boxes * BOX_BYTES;
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
-    cudaError_t e = cudaFuncSetAttribute(k_conv_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    using Kernel = void (*)(const ConvParams, const ExpandCfg, const CUtensorMap, const CUtensorMap);
+    const Kernel kernel = cfg.balanced ? (cfg.kblk == 2 ? k_conv_expand<2, true> : k_conv_expand<1, true>)
+                                       : (cfg.kblk == 2 ? k_conv_expand<2, false> : k_conv_expand<1, false>);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
     long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
+    if (cfg.balanced) {
+        static std::atomic<uint32_t> epoch{0};
+        grid = sm_count();
+        do cfg.epoch = epoch.fetch_add(1, std::memory_order_relaxed) + 1; while (cfg.epoch == 0);   // zero = a cleared flag
+    }
     if (cfg.w_res) grid = (grid / cfg.n_slices) * cfg.n_slices;   // n_work is a multiple of n_slices, so grid >= n_slices
-    e = nmhost::launch_pdl(k_conv_expand, static_cast<unsigned>(grid), THREADS, smem, st, q, cfg, tm_x, tm_y);
+    e = nmhost::launch_pdl(kernel, static_cast<unsigned>(grid), THREADS, smem, st, q, cfg, tm_x, tm_y);
     nmhost::count_launch(1);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 4): %s", cudaGetErrorString(e));

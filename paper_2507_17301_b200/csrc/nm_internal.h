@@ -117,6 +117,7 @@ nm_status_t launch_conv_slab(const ConvParams& p, const nm_plan_t* plan, cudaStr
 // nm_conv_expand.cu — variant 4
 bool expand_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 size_t expand_splitk_bytes(const ConvParams& p, int splits);   // scratch a split-K plan of this layer needs
+size_t expand_balanced_bytes(int bn);                          // scratch a balanced plan (split = -1) with this bn needs
 nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 
 // nm_conv_rowrun.cu — variant 5

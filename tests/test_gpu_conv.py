@@ -287,6 +287,48 @@ def test_split_k_plans(nm, integer):
         assert_conv_close(y.cpu().numpy(), yr)
 
 
+BALANCED = [
+    ConvShape("bal_few_items", 2, 14, 14, 256, 64, 3, 3, 1, 1, 1, 2, 4, 32),          # 4 items of 72 stages over all SMs: ~37 CTAs per item
+    ConvShape("bal_many_items", 8, 56, 56, 32, 256, 3, 3, 1, 1, 1, 2, 4, 64),         # 392 items of 9 stages: whole items and parts per CTA
+    ConvShape("bal_1x1_ragged", 3, 13, 13, 1024, 128, 1, 1, 1, 0, 1, 2, 4, 64),       # 507 pixels: ragged last block, 32 stages
+]
+
+
+@pytest.mark.parametrize("integer", [False, True], ids=["normal", "integer"])
+@pytest.mark.parametrize("s", BALANCED, ids=lambda s: s.name)
+def test_balanced_plans(nm, s, integer):
+    """Expanded-operand kernel with the (item, stage) pairs of the layer cut into one equal range per SM
+    (plan.split = -1): CTAs that share an item exchange partial sums through the handle's scratch."""
+    w, x, b = tensors_for(s, integer)
+    vr, ir, yr = oracle_layer(s, w, x, b)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    xd, bd = x.cuda(), b.cuda()
+    ran = 0
+    for bn, kblk, stages in ((64, 0, 0), (128, 2, 0), (32, 1, 2), (256, 0, 0)):
+        if s.c_out % bn:
+            continue
+        plan = nm.nm_plan_t()
+        plan.variant, plan.bn, plan.split, plan.kblk, plan.stages = 4, bn, -1, kblk, stages
+        need = nm.nm_plan_scratch_bytes(hnd, xd.shape, s.stride, s.pad, s.dil, plan)
+        assert need >= 128 * bn * 4
+        nm.nm_weights_reserve(hnd, need)
+        try:
+            for _ in range(3):                                # several launches: slots and flags are reused
+                y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
+        except nm.NmError as e:
+            if e.status == nm.NM_ERR_UNSUPPORTED:
+                continue                                      # e.g. K / 32 odd with two blocks per stage
+            raise
+        nm.nm_weights_check(hnd)
+        torch.cuda.synchronize()
+        ran += 1
+        if integer:
+            assert np.array_equal(y.cpu().numpy(), yr), (s.name, bn)
+        else:
+            assert_conv_close(y.cpu().numpy(), yr)
+    assert ran >= 2
+
+
 # Groups as wide as the input-channel axis (the paper's adaptive setting, Sec. 3.1: M may span all input
 # channels, N = (1 - sparsity) * M): every kernel that reads the tap table or the expanded weights takes them.
 LARGE_M = [
