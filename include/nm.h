@@ -188,8 +188,11 @@ nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int 
 
 /*
  * Scratch memory of a handle.  A plan that splits the reduction axis over several CTAs (variant 4
- * with split > 1) passes partial sums through scratch memory owned by the handle; nm_conv2d never
- * allocates, so the scratch must be there before such a plan is used.  nm_autotune reserves it for the
+ * with split > 1) or balances it over the SMs (split = -1: one slot of 128 x bn partial sums and eight
+ * flag words per SM) passes partial sums through scratch memory owned by the handle; nm_conv2d never
+ * allocates, so the scratch must be there before such a plan is used.  The scratch is cleared when it is
+ * reserved (the flag words must start at zero).  In balanced mode CTAs of one launch wait, with a bound,
+ * for flags raised by CTAs of lower index of the same launch (all CTAs of the launch fit the GPU at once).  nm_autotune reserves it for the
  * layers it tunes; a caller that brings a plan from elsewhere (a plan cache) asks for the size with
  * nm_plan_scratch_bytes (0 for plans that need none) and reserves it with nm_weights_reserve, which
  * allocates synchronously and keeps the larger of the old and new sizes.  Calls that use the same
