@@ -569,6 +569,34 @@ def main():
                               "finite": bool(torch.isfinite(last).all()),
                               "note": "conv backbone in dataflow order: stem, 3x3/2 max-pool, residual blocks with the "
                                       "shortcut addition fused into the block's last convolution"}
+            # the same step recorded once as a CUDA graph and replayed (no per-launch host work in the timed region)
+            try:
+                ref = last.clone()
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(graph, stream=side):
+                        g_last = chained_step()
+                torch.cuda.current_stream().wait_stream(side)
+                for _ in range(3):
+                    graph.replay()
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+                a.record()
+                for _ in range(args.steps):
+                    graph.replay()
+                b.record()
+                b.synchronize()
+                g_ms = a.elapsed_time(b) / args.steps
+                out["chained_graph"] = {"value": args.batch / (g_ms * 1e-3), "unit": UNIT, "ms_per_step": g_ms,
+                                        "same_output_as_launches": bool(torch.equal(g_last, ref)),
+                                        "note": "the chained step captured in one CUDA graph and replayed"}
+                for _s, hnd, *_r in state:
+                    nm.nm_weights_check(hnd)
+            except Exception as e:  # a capture the runtime refuses is reported, not fatal
+                out["chained_graph"] = {"unavailable": f"{type(e).__name__}: {e}"[:300]}
+                torch.cuda.synchronize()
 
         # cuDNN dense convolution on the same shapes (context, unpruned weights, TF32 allowed)
         try:

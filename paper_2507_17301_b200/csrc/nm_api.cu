@@ -371,6 +371,8 @@ nm_status_t nm_weights_check(const nm_weights_t* w, void* cuda_stream)
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_weights_check: %s", cudaGetErrorString(e));
     if (host[0] != 0) {
         cudaMemsetAsync(w->status, 0, 3 * sizeof(int), st);
+        // a balanced launch that gave up may have left flags raised at the start of the scratch
+        if (w->splitk) cudaMemsetAsync(w->splitk, 0, w->splitk_bytes < 16384 ? w->splitk_bytes : 16384, st);
         cudaStreamSynchronize(st);
         return nmhost::fail(static_cast<nm_status_t>(host[0]), "device-side wait expired (site %d, block %d)", host[1],
                             host[2]);

@@ -29,11 +29,11 @@
 // begins inside an item handles that part FIRST, stores the raw partial accumulator to its own
 // slot of the handle's scratch and raises a per-warp flag; the CTA whose range holds the item's
 // first stage handles it LAST, waits (bounded) for the flags of the others, adds their partial sums
-// to its accumulator and runs the normal epilogue.  Ranges are handed out from the end of the
+// to its accumulator, lowers the flags again (every flag has exactly one reader, so the scratch is
+// back in its cleared state when the launch ends and a recorded launch can be replayed) and runs
+// the normal epilogue.  Ranges are handed out from the end of the
 // layer to CTA 0 upwards, so a CTA only ever waits for CTAs with a lower index, whose first action
 // is the store it waits for.
-#include <atomic>
-
 #include "nm_internal.h"
 #include "nm_ptx.cuh"
 #include "nm_tmap.cuh"
@@ -64,7 +64,6 @@ struct ExpandCfg {
     int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
     int boxes;        // output staging boxes per epilogue warp: 2 for short reductions, 1 when the ring needs the room
     int balanced;     // 1: contiguous (item, stage) ranges per CTA, partial sums through per-CTA scratch slots
-    uint32_t epoch;   // balanced mode: value the flags of this launch carry
     long long n_work;
 };
 
@@ -300,7 +299,9 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         // balanced mode: this CTA's partial-sum slot (128 rows x bn) and its warps' flags, in the handle's scratch
         const uint32_t units = static_cast<uint32_t>(cfg.n_work) * static_cast<uint32_t>(cfg.n_sub);
         const size_t slot_floats = static_cast<size_t>(BM) * cfg.bn;
-        uint32_t* const flags = reinterpret_cast<uint32_t*>(p.splitk + slot_floats * gridDim.x);
+        // scratch layout: eight flag words per CTA first, then the slots
+        uint32_t* const flags = reinterpret_cast<uint32_t*>(p.splitk);
+        float* const slots = p.splitk + static_cast<size_t>(gridDim.x) * 8;
         const int my_row = q * 32 + lane;
         SegIter<BAL> it = make_iter<BAL>(cfg);
         Seg seg;
@@ -338,7 +339,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 for (uint32_t pos = first_pos + 1u; pos <= last_pos; ++pos) {
                     const uint32_t* f = flags + (gridDim.x - 1u - pos) * 8u + (warp - 4);
                     bool seen = false;
-                    for (uint32_t poll = 0; poll < kWaitPolls && !seen; ++poll) seen = ld_acquire_gpu(f) == cfg.epoch;
+                    for (uint32_t poll = 0; poll < kWaitPolls && !seen; ++poll) seen = ld_acquire_gpu(f) == 1u;
                     if (!seen) *abort_flag = 10;
                 }
                 if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
@@ -355,7 +356,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 if (publish) {
                     // raw partial sums of this thread's row; the slot is laid out [channel quad][row], so the 32
                     // lanes of a warp (32 consecutive rows) write 512 contiguous bytes per instruction
-                    float4* dst = reinterpret_cast<float4*>(p.splitk + slot_floats * blockIdx.x) +
+                    float4* dst = reinterpret_cast<float4*>(slots + slot_floats * blockIdx.x) +
                                   static_cast<size_t>(blk) * 8 * BM + my_row;
 #pragma unroll
                     for (int qq = 0; qq < 8; ++qq)
@@ -366,7 +367,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 }
                 if (finish) {
                     for (uint32_t pos = first_pos + 1u; pos <= last_pos; ++pos) {
-                        const float4* src = reinterpret_cast<const float4*>(p.splitk + slot_floats * (gridDim.x - 1u - pos)) +
+                        const float4* src = reinterpret_cast<const float4*>(slots + slot_floats * (gridDim.x - 1u - pos)) +
                                             static_cast<size_t>(blk) * 8 * BM + my_row;
                         float4 t4[8];
 #pragma unroll
@@ -429,7 +430,14 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 // every lane's stores are ordered before the flag the reading warp acquires
                 __threadfence();
                 __syncwarp();
-                if (lane == 0) st_release_gpu(flags + blockIdx.x * 8u + (warp - 4), cfg.epoch);
+                if (lane == 0) st_release_gpu(flags + blockIdx.x * 8u + (warp - 4), 1u);
+            }
+            if (finish) {
+                // this warp was the only reader of its counterparts' flags and has consumed their sums
+                __syncwarp();
+                if (lane == 0)
+                    for (uint32_t pos = first_pos + 1u; pos <= last_pos; ++pos)
+                        flags[(gridDim.x - 1u - pos) * 8u + (warp - 4)] = 0u;
             }
         }
         if (lane == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads; the writes complete with the grid
@@ -542,7 +550,6 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     cfg->n_work = ((p.pixels + BM - 1) / BM) * cfg->n_slices * splits;
     if (cfg->n_work >= (1ll << 31)) return false;
     cfg->balanced = 0;
-    cfg->epoch = 0;
     if (balanced) {
         // one range per SM; needs at least one (item, stage) unit per CTA and the per-CTA slots + flags in the scratch
         const long long units = cfg->n_work * cfg->n_sub;
@@ -597,11 +604,7 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
     long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    if (cfg.balanced) {
-        static std::atomic<uint32_t> epoch{0};
-        grid = sm_count();
-        do cfg.epoch = epoch.fetch_add(1, std::memory_order_relaxed) + 1; while (cfg.epoch == 0);   // zero = a cleared flag
-    }
+    if (cfg.balanced) grid = sm_count();
     if (cfg.w_res) grid = (grid / cfg.n_slices) * cfg.n_slices;   // n_work is a multiple of n_slices, so grid >= n_slices
     e = nmhost::launch_pdl(kernel, static_cast<unsigned>(grid), THREADS, smem, st, q, cfg, tm_x, tm_y);
     nmhost::count_launch(1);
