@@ -103,7 +103,10 @@ WORKLOAD = {"depth": 50, "n": 2, "m": 4, "tile": 64}   # the headline configurat
 
 
 def workload(batch: int):
-    layers = inputs.resnet_conv_stack(WORKLOAD["depth"], batch, WORKLOAD["n"], WORKLOAD["m"], tile_t=WORKLOAD["tile"])
+    if WORKLOAD.get("net") == "mobilenet_v2":
+        layers = inputs.mobilenet_v2_pointwise(batch, WORKLOAD["n"], WORKLOAD["m"], tile_t=WORKLOAD["tile"])
+    else:
+        layers = inputs.resnet_conv_stack(WORKLOAD["depth"], batch, WORKLOAD["n"], WORKLOAD["m"], tile_t=WORKLOAD["tile"])
     r = WORKLOAD.get("adaptive")
     if r is not None:
         # the paper's adaptive setting (Sec. 3.1): a group spans a layer's input channels, N = (1 - sparsity) * M
@@ -114,6 +117,8 @@ def workload(batch: int):
 
 def workload_name(batch: int) -> str:
     pat = f"{WORKLOAD['n']}of{WORKLOAD['m']}" if WORKLOAD.get("adaptive") is None else f"adaptiveM_sparsity{WORKLOAD['adaptive']}"
+    if WORKLOAD.get("net") == "mobilenet_v2":
+        return f"mobilenet_v2_pointwise_convs_b{batch}_224_{pat}"
     return f"resnet{WORKLOAD['depth']}_conv_stack_b{batch}_224_{pat}"
 
 
@@ -310,6 +315,8 @@ def main():
     ap.add_argument("--split", type=int, default=0, help="with --variant: the plan's split field")
     ap.add_argument("--kblk", type=int, default=0, help="with --variant: 32-column blocks per pipeline stage")
     ap.add_argument("--depth", type=int, default=50, choices=[18, 34, 50, 101, 152], help="ResNet depth of the conv stack")
+    ap.add_argument("--net", default="resnet", choices=["resnet", "mobilenet_v2"],
+                    help="mobilenet_v2: its pointwise (1x1) convolutions only, the layers the paper prunes there")
     ap.add_argument("--nm", default="2:4", help="N:M pattern of the pruned layers, e.g. 1:4 or 2:8")
     ap.add_argument("--tile", type=int, default=64, help="pruning tile width T")
     ap.add_argument("--adaptive", type=float, default=None,
@@ -319,7 +326,7 @@ def main():
     ap.add_argument("--load-plans", default=None, help="use the plans of this JSON file instead of auto-tuning")
     args = ap.parse_args()
     WORKLOAD.update(depth=args.depth, n=int(args.nm.split(":")[0]), m=int(args.nm.split(":")[1]), tile=args.tile,
-                    adaptive=args.adaptive)
+                    adaptive=args.adaptive, net=args.net)
     if args.impl == "reference":
         return run_reference(args)
     if args.warmup < 3:
@@ -528,7 +535,7 @@ def main():
 
         # the same layers chained as the network's dataflow: stem -> max-pool -> residual blocks, every
         # layer reading its predecessor's output, shortcut additions fused into the last conv of a block
-        if not args.layer:
+        if not args.layer and args.net == "resnet":
             idx = {s.name: i for i, (s, *_rest) in enumerate(state)}
             pool_out = torch.empty((args.batch, state[1][0].h, state[1][0].w, 64), dtype=torch.float32, device=dev)
             prefixes = []

@@ -123,6 +123,7 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     p->rel2 = w->v2_ok ? w->rel2 : nullptr;
     p->v2_kc = w->v2_kc; p->v2_s = w->v2_s; p->v2_chunks = w->v2_chunks;
     p->wx = w->wx;
+    p->wx_rows = w->wx_rows;
     p->splitk = w->splitk;
     p->splitk_bytes = w->splitk_bytes;
     return NM_OK;
@@ -172,8 +173,15 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     a.variant = 5;                          // row-run kernel (few input channels)
     if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, &a)) out.push_back(a);
     std::memset(&a, 0, sizeof(a));
+    // channel widths of a work item for the expanded-operand kernel: the usual three, plus the whole (padded)
+    // channel count and 32 for layers whose channel count is not a multiple of 64
+    std::vector<int> widths = {64, 128, 256};
+    if (p.wx_rows % 64 != 0) {
+        if (p.wx_rows <= 256) widths.push_back(p.wx_rows);
+        if (p.wx_rows != 32) widths.push_back(32);
+    }
     for (int split : {0, 1}) {              // expanded-operand kernel: weights resident where they fit / streamed,
-        for (int bn : {64, 128, 256}) {     // one or two 32-column blocks per pipeline stage
+        for (int bn : widths) {             // one or two 32-column blocks per pipeline stage
             for (int kblk : {1, 2}) {
                 a.variant = 4; a.bn = bn; a.stages = 0; a.split = split; a.kblk = kblk;
                 if (nmhost::expand_plan_ok(p, &a)) out.push_back(a);

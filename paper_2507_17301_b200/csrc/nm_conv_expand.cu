@@ -185,11 +185,11 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 const int slice = static_cast<int>(blockIdx.x % static_cast<uint32_t>(cfg.n_slices));
                 mbar_arrive_expect_tx(smem_u32(&s_wres), static_cast<uint32_t>(n_blk32) * static_cast<uint32_t>(cfg.bn) * 128u);
                 for (int c = 0; c < n_blk32; ++c)
-                    bulk_load_1d(wres + c * cfg.b_bytes, p.wx + (static_cast<size_t>(c) * p.c_out + slice * cfg.bn) * 32,
+                    bulk_load_1d(wres + c * cfg.b_bytes, p.wx + (static_cast<size_t>(c) * p.wx_rows + slice * cfg.bn) * 32,
                                  static_cast<uint32_t>(cfg.bn) * 128u, smem_u32(&s_wres));
             }
             const uint32_t w_bytes = static_cast<uint32_t>(cfg.bn) * 128u;
-            const size_t w_step = static_cast<size_t>(p.c_out) * 32;   // floats between two 32-column blocks
+            const size_t w_step = static_cast<size_t>(p.wx_rows) * 32;   // floats between two 32-column blocks
             RingPos rp;
             SegIter<BAL> it = make_iter<BAL>(cfg);
             Seg seg;
@@ -321,7 +321,8 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const int res_rows = p.pixels - box_pix < 32 ? static_cast<int>(p.pixels - box_pix) : 32;
             const float* res_base = res_pass ? p.residual + box_pix * p.c_out + slice * cfg.bn : nullptr;
             float4 rv[8];
-            if (res_pass && half < n_blk) load_residual_box(rv, res_base + half * 32, p.c_out, res_rows, lane);
+            const int cols_left = p.c_out - slice * cfg.bn;   // channels of this slice that exist (may end inside a box)
+            if (res_pass && half < n_blk) load_residual_box(rv, res_base + half * 32, p.c_out, res_rows, lane, cols_left - half * 32);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
@@ -396,7 +397,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 for (int qq = 0; qq < 8; ++qq) {
                     float o[4];
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
+                    if (p.bias && blk * 32 + qq * 4 < cols_left) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
                     o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                     o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                     o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
@@ -412,7 +413,8 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 if (res_pass) {
                     __syncwarp();
                     apply_residual_box(box, rv, p.relu, lane);
-                    if (blk + 2 < n_blk) load_residual_box(rv, res_base + (blk + 2) * 32, p.c_out, res_rows, lane);
+                    if (blk + 2 < n_blk)
+                        load_residual_box(rv, res_base + (blk + 2) * 32, p.c_out, res_rows, lane, cols_left - (blk + 2) * 32);
                 }
                 fence_proxy_async();
                 __syncwarp();
@@ -496,7 +498,11 @@ int sm_count()
 bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
 {
     if (!p.wx || !nmtm::available()) return false;
-    if (p.c_in % 32 != 0 || p.c_out % 32 != 0) return false;
+    // whole 32-channel input blocks, or a pointwise layer whose last block the TMA unit fills up with zeros;
+    // output channels in whole float4s (the expanded weights are padded to 32-row blocks)
+    const bool pointwise = p.kh == 1 && p.kw == 1;
+    if (p.c_in % 32 != 0 && !(pointwise && p.c_in % 4 == 0)) return false;
+    if (p.c_out % 4 != 0 || p.wx_rows < p.c_out || p.wx_rows % 32 != 0) return false;
     if (!nmtm::im2col_geometry_ok(p)) return false;
     if (static_cast<long long>(p.batch) * p.h * p.w * p.c_in * 4 < 131072) return false;
     if (p.pixels >= (1ll << 31) - BM) return false;
@@ -505,17 +511,18 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
         bn = plan->bn;
     } else {
         for (int cand : {128, 256, 64, 96, 32, 160, 192, 224})
-            if (cand <= p.c_out && p.c_out % cand == 0) { bn = cand; break; }
+            if (cand <= p.wx_rows && p.wx_rows % cand == 0) { bn = cand; break; }
     }
-    if (bn < 32 || bn > 256 || bn % 32 != 0 || p.c_out % bn != 0) return false;
+    if (bn < 32 || bn > 256 || bn % 32 != 0 || p.wx_rows % bn != 0) return false;
     cfg->bn = bn;
-    cfg->n_slices = p.c_out / bn;
+    cfg->n_slices = p.wx_rows / bn;
     cfg->b_bytes = ((bn * 128 + 1023) / 1024) * 1024;
     const int splits = plan && plan->split > 1 ? plan->split : 1;
     const bool balanced = plan && plan->split == -1;
-    if (splits > 8 || (p.k / 32) % splits != 0) return false;
+    const int k_blocks = (p.k + 31) / 32;   // the last block of a pointwise layer may be partly zero fill
+    if (splits > 8 || k_blocks % splits != 0) return false;
     cfg->ksplit = splits;
-    const int blk32 = (p.k / 32) / splits;   // 32-column blocks per work item
+    const int blk32 = k_blocks / splits;   // 32-column blocks per work item
     const int kblk = plan && plan->kblk > 0 ? plan->kblk : 1;
     if (kblk > 2 || blk32 % kblk != 0) return false;
     cfg->kblk = kblk;

@@ -31,7 +31,8 @@ struct nm_weights {
     // Expanded layout (variant 4): the pruned matrix back in dense shape, zeros in the pruned columns.
     float* splitk;       // scratch for split-K partial sums (variant 4), allocated by nm_autotune; may be NULL
     size_t splitk_bytes;
-    float* wx;           // [ceil(k / 32)][c_out][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
+    float* wx;           // [ceil(k / 32)][wx_rows][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
+    int wx_rows;         // c_out rounded up to a multiple of 32 (the rows past c_out are zero)
 };
 
 // Geometry handed to the convolution kernels.
@@ -56,6 +57,7 @@ struct ConvParams {
     int v2_kc, v2_s, v2_chunks;
     // expanded layout (variant 4)
     const float* wx;
+    int wx_rows;
     // split-K scratch of the handle (variant 4 with plan.split > 1)
     float* splitk;
     size_t splitk_bytes;

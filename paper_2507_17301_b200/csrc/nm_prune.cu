@@ -145,7 +145,7 @@ __global__ void k_build_slab(const float* __restrict__ values, const uint16_t* _
 // stored as the shared-memory image the tensor core reads: blocks of 32 columns, inside a block
 // one 128-byte row per output channel whose 16-byte pieces are XOR-ed with (o % 8) (the 128-byte
 // swizzle), so that any run of channels starting at a multiple of 8 is one contiguous bulk copy.
-__global__ void k_expand(const float* __restrict__ values, const uint16_t* __restrict__ indices, int c_out, int kk,
+__global__ void k_expand(const float* __restrict__ values, const uint16_t* __restrict__ indices, int rows, int kk,
                          int tile_t, float* __restrict__ wx)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -153,7 +153,7 @@ __global__ void k_expand(const float* __restrict__ values, const uint16_t* __res
     if (j >= kk) return;
     const int col = indices[static_cast<size_t>(o / tile_t) * kk + j];
     const int blk = col >> 5, kc = col & 31;
-    wx[(static_cast<size_t>(blk) * c_out + o) * 32 + ((((kc >> 2) ^ (o & 7)) << 2) | (kc & 3))] =
+    wx[(static_cast<size_t>(blk) * rows + o) * 32 + ((((kc >> 2) ^ (o & 7)) << 2) | (kc & 3))] =
         nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
 }
 
@@ -262,10 +262,13 @@ nm_status_t build_slab_layout(nm_weights* h, cudaStream_t st)
 nm_status_t build_expanded_layout(nm_weights* h, cudaStream_t st)
 {
     h->wx = nullptr;
-    // only shapes the kernels that read it take: 32-channel output blocks, and either whole
-    // 32-column slabs (expanded-operand kernel) or a short reduction axis (row-run kernel)
-    if (h->c_out % 32 != 0 || h->kk == 0 || (h->c_in % 32 != 0 && h->k > 512)) return NM_OK;
-    const size_t bytes = static_cast<size_t>((h->k + 31) / 32) * h->c_out * 32 * sizeof(float);
+    h->wx_rows = 0;
+    // only shapes the kernels that read it take: output channels in whole float4s (rows are padded with
+    // zeros to blocks of 32), and either whole 32-column slabs (expanded-operand kernel) or a short
+    // reduction axis (row-run kernel, pointwise layers)
+    if (h->c_out % 4 != 0 || h->kk == 0 || (h->c_in % 32 != 0 && h->k > 512)) return NM_OK;
+    h->wx_rows = (h->c_out + 31) / 32 * 32;
+    const size_t bytes = static_cast<size_t>((h->k + 31) / 32) * h->wx_rows * 32 * sizeof(float);
     if (cudaMalloc(&h->wx, bytes) != cudaSuccess) {
         (void)cudaGetLastError();
         h->wx = nullptr;
@@ -274,7 +277,7 @@ nm_status_t build_expanded_layout(nm_weights* h, cudaStream_t st)
     cudaError_t e = cudaMemsetAsync(h->wx, 0, bytes, st);
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "expanded layout memset: %s", cudaGetErrorString(e));
     const dim3 grid((h->kk + 127) / 128, h->c_out);
-    k_expand<<<grid, 128, 0, st>>>(h->values, h->indices, h->c_out, h->kk, h->tile_t, h->wx);
+    k_expand<<<grid, 128, 0, st>>>(h->values, h->indices, h->wx_rows, h->kk, h->tile_t, h->wx);
     count_launch(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "expanded layout kernel: %s", cudaGetErrorString(e));

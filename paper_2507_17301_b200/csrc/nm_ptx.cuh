@@ -270,14 +270,17 @@ __device__ __forceinline__ void tma_prefetch_desc(const void* tmap)
 // the residual (a thread reading its own row piece by piece would touch 32 lines per instruction).
 //   res       first residual element of the box's first row; row pitch c_out floats
 //   rows      rows of the box that exist (the last block of a layer may be ragged)
-__device__ __forceinline__ void load_residual_box(float4 (&rv)[8], const float* res, int c_out, int rows, int lane)
+//   cols      channels of the box that exist (32 unless the layer's channel count is not a multiple of 32)
+__device__ __forceinline__ void load_residual_box(float4 (&rv)[8], const float* res, int c_out, int rows, int lane,
+                                                  int cols = 32)
 {
     const int piece = lane & 7;
+    const bool col_ok = piece * 4 < cols;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int r = i * 4 + (lane >> 3);
-        rv[i] = r < rows ? __ldg(reinterpret_cast<const float4*>(res + static_cast<size_t>(r) * c_out) + piece)
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
+        rv[i] = (r < rows && col_ok) ? __ldg(reinterpret_cast<const float4*>(res + static_cast<size_t>(r) * c_out) + piece)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
 __device__ __forceinline__ void apply_residual_box(uint32_t box, const float4 (&rv)[8], int relu, int lane)

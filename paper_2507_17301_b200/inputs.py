@@ -181,3 +181,34 @@ def resnet_conv_stack(depth: int, batch: int, n_keep: int, m_group: int, tile_t:
             hw = hw_out
             c_prev = 4 * width
     return layers
+
+
+def mobilenet_v2_pointwise(batch: int, n_keep: int, m_group: int, tile_t: int = 16, image: int = 224):
+    """The pointwise (1x1) convolutions of MobileNet-V2 in network order: per inverted-residual block the
+    expansion (absent where the expansion factor is 1) and the linear projection, then the final 1x1
+    convolution.  These are the layers the paper prunes in this network (Sec. 4.5: the depthwise
+    convolutions stay dense and are not part of the pruned path), so the 3x3 stem and the depthwise
+    layers only appear here through the map sizes they produce.
+
+    Standard architecture (Sandler et al. 2018): stem 3x3/2 to 32 channels, blocks given as
+    (expansion t, channels c, repeats n, stride s), the stride on the first repeat's depthwise layer.
+    Several channel counts (16, 24, 144, ...) are not multiples of 32: those layers exercise the general kernels.
+    """
+    table = ((1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2), (6, 96, 3, 1), (6, 160, 3, 2), (6, 320, 1, 1))
+    mk = dict(n_keep=n_keep, m_group=m_group, tile_t=tile_t)
+    layers = []
+    hw = (image + 2 - 3) // 2 + 1   # after the stem: 112
+    c_prev = 32
+    for bi, (t, c, n, s) in enumerate(table):
+        for ri in range(n):
+            stride = s if ri == 0 else 1
+            pre = f"b{bi + 1}r{ri + 1}"
+            hidden = c_prev * t
+            if t != 1:
+                layers.append(ConvShape(pre + "_expand", batch, hw, hw, c_prev, hidden, **mk))      # followed by ReLU6 in the network; ReLU here
+            hw = (hw + 2 - 3) // stride + 1                                                            # the depthwise 3x3 in between
+            layers.append(ConvShape(pre + "_project", batch, hw, hw, hidden, c, relu=False, **mk))   # linear bottleneck
+            c_prev = c
+    layers.append(ConvShape("last_1x1", batch, hw, hw, c_prev, 1280, **mk))
+    return layers
+

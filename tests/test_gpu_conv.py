@@ -182,6 +182,28 @@ def test_window_shapes_integer_exact(nm, s):
     _run(nm, s, integer=True, need_variant=[6])
 
 
+# pointwise layers whose channel counts are not multiples of 32 (MobileNet-like): the expanded-operand kernel lets
+# the TMA unit zero-fill the last input block and pads the weight rows
+POINTWISE = [
+    ConvShape("pw_cin24", 2, 56, 56, 24, 144, 1, 1, 1, 0, 1, 2, 4, 16),
+    ConvShape("pw_cout24", 2, 56, 56, 96, 24, 1, 1, 1, 0, 1, 2, 4, 8),
+    ConvShape("pw_cin144_cout24", 2, 40, 40, 144, 24, 1, 1, 1, 0, 1, 2, 4, 8),
+    ConvShape("pw_cin16_cout96", 1, 112, 112, 16, 96, 1, 1, 1, 0, 1, 2, 4, 16),
+    ConvShape("pw_cout16", 1, 112, 112, 32, 16, 1, 1, 1, 0, 1, 2, 4, 16),
+    ConvShape("pw_cout40_stride2", 2, 57, 57, 48, 40, 1, 1, 2, 0, 1, 1, 4, 8),       # strided, ragged pixel tail (841 pixels)
+]
+
+
+@pytest.mark.parametrize("s", POINTWISE, ids=lambda s: s.name)
+def test_pointwise_ragged_channels(nm, s):
+    _run(nm, s, need_variant=[1, 4])
+
+
+@pytest.mark.parametrize("s", POINTWISE, ids=lambda s: s.name)
+def test_pointwise_ragged_channels_integer_exact(nm, s):
+    _run(nm, s, integer=True, need_variant=[4])
+
+
 # pair kernel (variant 7): clusters of two CTAs share one 256-pixel x bn MMA
 PAIR = [
     ConvShape("pair_one", 1, 16, 16, 128, 256, 3, 3, 1, 1, 1, 2, 4, 64),              # 2 pixel blocks: one pair, one item

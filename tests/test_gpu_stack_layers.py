@@ -17,6 +17,9 @@ LAYERS = [(50, "stem7x7"), (50, "s1b1_c3"), (50, "s1b1_c2"), (50, "s2b1_c2"), (5
           (50, "s4b2_c1"), (50, "s4b2_c2"),
           # basic-block network (ResNet-34): strided 3x3 that doubles the channels, 3x3 at 28x28
           (34, "s2b1_c1"), (34, "s2b2_c2")]
+# pointwise layers of MobileNet-V2 (tile width 16): channel counts that are not multiples of 32 on either
+# side (general kernels), the widest expansion, the last 1x1
+MOBILE_LAYERS = ["b1r1_project", "b2r2_expand", "b3r1_project", "b5r2_expand", "b6r2_project", "last_1x1"]
 IMAGES = (0, 37, 63)
 
 
@@ -58,3 +61,34 @@ def test_stack_layer_sampled_images(nm, stack, depth, name):
     yc = y.cpu()
     assert torch.isfinite(yc).all()
     assert (yc.abs().amax(dim=(1, 2, 3)) > 0).all()
+
+
+@pytest.fixture(scope="module")
+def mobile_stack():
+    return {s.name: (i, s) for i, s in enumerate(inputs.mobilenet_v2_pointwise(64, 2, 4, tile_t=16))}
+
+
+@pytest.mark.parametrize("name", MOBILE_LAYERS)
+def test_mobilenet_pointwise_sampled_images(nm, mobile_stack, name):
+    li, s = mobile_stack[name]
+    w = inputs.make_weights(s, li)
+    b = inputs.make_bias(s, li)
+    g = torch.Generator().manual_seed(1 + 1000 * li)
+    x = torch.randn((s.batch, s.h, s.w, s.c_in), generator=g)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    v, i = nm.nm_weights_export(hnd)
+    vr, ir = oracle.prune(w.numpy(), s.n_keep, s.m_group, s.tile_t)
+    assert_prune_bit_exact(v.cpu().numpy(), i.cpu().numpy(), vr, ir)
+    xd, bd = x.cuda(), b.cuda()
+    plan, ms = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)
+    assert ms > 0
+    for use in (plan, None):                                  # the tuned plan and the library default
+        y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=use)
+        nm.nm_weights_check(hnd)
+        torch.cuda.synchronize()
+        for n in IMAGES[:2]:
+            yr = oracle.conv2d(vr, ir, s.kh, s.kw, s.c_in, s.tile_t, x[n:n + 1].numpy(), (s.stride,) * 2, (s.pad,) * 2,
+                               (s.dil,) * 2, b.numpy(), s.relu)
+            assert_conv_close(y[n:n + 1].cpu().numpy(), yr)
+        assert torch.isfinite(y).all()
+

@@ -36,3 +36,21 @@ def test_resnet_stacks_have_the_published_conv_counts_and_flops():
     assert abs(sum(s.pixels * s.c_out * s.k for s in r18) / 1e9 - 1.81) < 0.05
     assert abs(sum(s.pixels * s.c_out * s.k for s in r34) / 1e9 - 3.66) < 0.05
     assert (r34[-1].ho, r34[-1].c_out, r34[-1].kh) == (7, 512, 3)
+
+
+def test_mobilenet_v2_pointwise_shapes():
+    layers = inputs.mobilenet_v2_pointwise(1, 2, 4)
+    assert len(layers) == 34                                   # 16 expansions + 17 projections + the last 1x1
+    assert all(s.kh == 1 and s.kw == 1 and s.stride == 1 for s in layers)
+    assert (layers[0].c_in, layers[0].c_out, layers[0].h) == (32, 16, 112)
+    assert (layers[-1].c_in, layers[-1].c_out, layers[-1].h) == (320, 1280, 7)
+    # a projection's input is its block's expansion output; the chain of block outputs is 16, 24, ..., 320
+    outs = [s.c_out for s in layers if s.name.endswith("_project")]
+    assert outs == [16, 24, 24, 32, 32, 32, 64, 64, 64, 64, 96, 96, 96, 160, 160, 160, 320]
+    for a, b in zip(layers, layers[1:]):
+        if a.name.endswith("_expand"):
+            assert b.name.endswith("_project") and b.c_in == a.c_out == 6 * a.c_in
+    # multiply-accumulates of the dense pointwise layers at 224 x 224 (a check of the map sizes)
+    macs = sum(s.ho * s.wo * s.c_in * s.c_out for s in layers)
+    assert 250e6 < macs < 300e6
+
