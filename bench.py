@@ -428,6 +428,32 @@ def main():
     }
 
     if rank == 0 and not args.no_extras and world == 1:
+        # the same step recorded once as a CUDA graph and replayed: what the GPU does when the host's launch
+        # calls are out of the way (matters for networks of small layers)
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    step()
+            torch.cuda.current_stream().wait_stream(side)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+            a.record()
+            for _ in range(args.steps):
+                graph.replay()
+            b.record()
+            b.synchronize()
+            g_ms = a.elapsed_time(b) / args.steps
+            out["graph_replay"] = {"value": args.batch / (g_ms * 1e-3), "unit": UNIT, "ms_per_step": g_ms,
+                                   "note": "the timed step captured in one CUDA graph and replayed"}
+            del graph
+        except Exception as e:
+            out["graph_replay"] = {"unavailable": f"{type(e).__name__}: {e}"[:300]}
+            torch.cuda.synchronize()
         # tensor roof: the measured bf16 GEMM peak scaled by the nominal TF32 : bf16 ratio; the library
         # TF32 GEMM timed here is context
         tf32_peak = pk["bf16_tflops"] * TF32_OVER_BF16
@@ -445,20 +471,41 @@ def main():
             xs = [x] + [x.clone() for _ in range(n_sets - 1)]
             ys = [y] + [torch.empty_like(y) for _ in range(n_sets - 1)]
             launches = max(20, 2 * n_sets)
+
+            def burst():
+                for k in range(launches):
+                    nm.nm_conv2d(hnd, xs[k % n_sets], s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu,
+                                 y=ys[k % n_sets], plan=plan)
+
+            # the burst is recorded once as a CUDA graph and replayed, so that small layers are timed at the
+            # GPU's pace and not at the pace of the host's launch calls; if the capture is refused the burst
+            # is launched directly
+            replay = burst
+            try:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(graph, stream=side):
+                        burst()
+                torch.cuda.current_stream().wait_stream(side)
+                replay = graph.replay
+                per_layer_mode = "graph replay"
+            except Exception:
+                torch.cuda.synchronize()
+                per_layer_mode = "direct launches"
             samples = []
             for rep in range(3):
                 for k in range(n_sets):   # also evicts what the previous repetition left in L2 in order
                     nm.nm_conv2d(hnd, xs[k], s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=ys[k], plan=plan)
                 a, b = torch.cuda.Event(True), torch.cuda.Event(True)
                 a.record()
-                for k in range(launches):
-                    nm.nm_conv2d(hnd, xs[k % n_sets], s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu,
-                                 y=ys[k % n_sets], plan=plan)
+                replay()
                 b.record()
                 b.synchronize()
                 samples.append(a.elapsed_time(b) / launches)
             per.append(samples)
-            del xs, ys
+            del replay, xs, ys
         table, t_roof_sum = [], 0.0
         for (s, hnd, x, bias, y, plan), ts in zip(state, per):
             ms = statistics.median(ts)
@@ -475,6 +522,7 @@ def main():
         out["stack_roofline_note"] = ("sum over layers of max(kept FLOPs / TF32 peak, algorithmic bytes / HBM peak) "
                                       "divided by the measured time of a step")
         out["per_layer"] = table
+        out["per_layer_mode"] = per_layer_mode
         # roofline object: the kernel that takes the largest share of a step, over all its launches
         by_kernel = {}
         for (s, hnd, x, bias, y, plan), row in zip(state, table):
@@ -502,7 +550,8 @@ def main():
             "useful_tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12,
             "time_frac_of_layer_rooflines": d["roof_ms"] / d["ms"],   # some of its layers are tensor-bound, not HBM-bound
             "note": "algorithmic bytes of the layers this kernel runs / their summed launch times (per layer: median of 3 runs "
-                    "of >= 20 back-to-back launches on rotating buffers larger than twice the L2)",
+                    "of >= 20 back-to-back launches, recorded as a CUDA graph and replayed, on rotating buffers larger "
+                    "than twice the L2)",
         }
 
         # the same stack restricted to the kernels that gather only the retained columns (variants 1-3:
