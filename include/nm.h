@@ -66,8 +66,9 @@ typedef struct nm_weights nm_weights_t;
  *                least 128 KiB);
  *            4 = expanded-operand kernel (persistent; the slab feeds the tensor core directly and
  *                zero weights stand for the pruned columns: M/N times the kept FLOPs, no
- *                per-element work; needs c_in % 32 == 0, c_out % 32 == 0, an input of at least
- *                128 KiB; any tile_t, any N:M);
+ *                per-element work; needs c_in % 32 == 0 (pointwise layers, kh = kw = 1: c_in % 4 == 0,
+ *                the last 32-channel block is filled up with zeros), c_out % 4 == 0, an input of at
+ *                least 128 KiB; any tile_t, any N:M);
  *            5 = row-run kernel for few input channels (c_in % 32 != 0, dil_w = 1, output rows of
  *                at most 128 pixels, K <= 512, c_out % 32 == 0 and <= 256, w * c_in * 4 a multiple
  *                of 16).
@@ -80,7 +81,8 @@ typedef struct nm_weights nm_weights_t;
  *                halves the shared-memory traffic per FLOP on reduction-heavy layers (needs the
  *                conditions of variant 4, bn 128 or 256, c_out % bn == 0).
  *   bn       output channels per CTA / work item (variants 2, 3: a multiple of tile_t; variant 4: a
- *            multiple of 32 up to 256; variant 6 likewise; variant 7: 128 or 256), 0 = default
+ *            multiple of 32 up to 256 that divides c_out rounded up to a multiple of 32; variant 6: a multiple
+ *            of 32 up to 256 that divides c_out; variant 7: 128 or 256), 0 = default
  *   stages   depth of the shared-memory ring, 0 = default
  *   split    variant 2: 1 = cp.async producer, 2 = direct-store epilogue; variant 4: 0 = keep a CTA's weight
  *            slice resident in shared memory when it fits, 1 = stream the weights with the activations,
