@@ -322,12 +322,13 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const float* res_base = res_pass ? p.residual + box_pix * p.c_out + slice * cfg.bn : nullptr;
             float4 rv[8];
             const int cols_left = p.c_out - slice * cfg.bn;   // channels of this slice that exist (may end inside a box)
+            const int o0 = slice * cfg.bn;
+            float bias_next = half < n_blk ? bias_lane_load(p.bias, o0 + half * 32, p.c_out, lane) : 0.f;   // first block's bias
             if (res_pass && half < n_blk) load_residual_box(rv, res_base + half * 32, p.c_out, res_rows, lane, cols_left - half * 32);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
-            const int o0 = slice * cfg.bn;
             // positions (of the equal ranges) that hold the rest of this item: first_pos + 1 .. last_pos
             uint32_t first_pos = 0, last_pos = 0;
             if (finish) {
@@ -393,11 +394,12 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 const uint32_t stage_row = box + lane * 128;
                 // with a shortcut input the activation waits for the second pass below
                 const int relu_now = res_pass ? 0 : p.relu;
+                const float bias_cur = bias_next;
+                if (blk + 2 < n_blk) bias_next = bias_lane_load(p.bias, o0 + (blk + 2) * 32, p.c_out, lane);   // a block ahead
 #pragma unroll
                 for (int qq = 0; qq < 8; ++qq) {
                     float o[4];
-                    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (p.bias && blk * 32 + qq * 4 < cols_left) bv = __ldg(reinterpret_cast<const float4*>(p.bias + o0 + blk * 32) + qq);
+                    const float4 bv = bias_quad(bias_cur, qq);
                     o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
                     o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
                     o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;

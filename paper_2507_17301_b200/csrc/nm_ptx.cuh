@@ -264,6 +264,20 @@ __device__ __forceinline__ void tma_prefetch_desc(const void* tmap)
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
 
+// Bias of a 32-channel block held one value per lane (lane l: channel first + l, zero past `c_out` or without a
+// bias), fetched ahead of the wait for the accumulator so that its latency is off the epilogue's critical path;
+// bias_quad() hands a thread the four values of channel quad `qq` by shuffles.
+__device__ __forceinline__ float bias_lane_load(const float* bias, int first, int c_out, int lane)
+{
+    const int ch = first + lane;
+    return (bias != nullptr && ch < c_out) ? __ldg(bias + ch) : 0.f;
+}
+__device__ __forceinline__ float4 bias_quad(float bias_lane, int qq)
+{
+    return make_float4(__shfl_sync(0xFFFFFFFFu, bias_lane, qq * 4 + 0), __shfl_sync(0xFFFFFFFFu, bias_lane, qq * 4 + 1),
+                       __shfl_sync(0xFFFFFFFFu, bias_lane, qq * 4 + 2), __shfl_sync(0xFFFFFFFFu, bias_lane, qq * 4 + 3));
+}
+
 // Adds the shortcut input to a staged 32-pixel x 32-channel output box (128-byte-swizzled rows) and
 // applies the activation, one warp per box.  The lanes walk the box four rows at a time, eight
 // 16-byte pieces per row, so that every global load instruction reads four full 128-byte lines of
