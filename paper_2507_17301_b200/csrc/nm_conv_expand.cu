@@ -194,21 +194,35 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             SegIter<BAL> it = make_iter<BAL>(cfg);
             Seg seg;
             while (!aborted(abort_flag) && it.next(seg)) {
+                // The item's coordinates, with the divisions the common cases do not need left out: this thread
+                // issues the kernel's first load only after them.
                 const uint32_t work = seg.work;
-                const int slice = static_cast<int>(work % static_cast<uint32_t>(cfg.n_slices));
-                const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
-                const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
-                const uint32_t pix0 = (rest / static_cast<uint32_t>(cfg.ksplit)) * BM;
+                uint32_t slice = 0, rest = work, ks = 0;
+                if (cfg.n_slices > 1) {
+                    rest = work / static_cast<uint32_t>(cfg.n_slices);
+                    slice = work - rest * static_cast<uint32_t>(cfg.n_slices);
+                }
+                if (cfg.ksplit > 1) {
+                    const uint32_t pb = rest / static_cast<uint32_t>(cfg.ksplit);
+                    ks = rest - pb * static_cast<uint32_t>(cfg.ksplit);
+                    rest = pb;
+                }
+                const uint32_t pix0 = rest * BM;
                 const int n0 = static_cast<int>(pix0 / static_cast<uint32_t>(hw));
                 const int rem = static_cast<int>(pix0 - static_cast<uint32_t>(n0) * static_cast<uint32_t>(hw));
                 const int oh0 = rem / p.wo, ow0 = rem - oh0 * p.wo;
                 const int w0 = ow0 * p.stride_w - p.pad_w, h0 = oh0 * p.stride_h - p.pad_h;
                 // first 32-column block of this item's share of the reduction axis
-                const int c0 = ks * n_blk32 + seg.sb * KBLK;
-                const int tap0 = (c0 * 32) / p.c_in;
+                const int c0 = static_cast<int>(ks) * n_blk32 + seg.sb * KBLK;
                 const float* wsrc = p.wx + static_cast<size_t>(slice) * cfg.bn * 32 + static_cast<size_t>(c0) * w_step;
-                int ch = c0 * 32 - tap0 * p.c_in, tw = tap0 % p.kw;
-                int off_w = tw * p.dil_w, off_h = (tap0 / p.kw) * p.dil_h;
+                int ch = 0, tw = 0, off_w = 0, off_h = 0;
+                if (c0 != 0) {
+                    const int tap0 = (c0 * 32) / p.c_in, th = tap0 / p.kw;
+                    ch = c0 * 32 - tap0 * p.c_in;
+                    tw = tap0 - th * p.kw;
+                    off_w = tw * p.dil_w;
+                    off_h = th * p.dil_h;
+                }
                 for (int c = seg.sb; c < seg.se; ++c) {
                     if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_free[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
