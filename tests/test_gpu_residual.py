@@ -17,7 +17,9 @@ SHAPES = [
     ConvShape("res_3x3_window", 2, 28, 28, 64, 64, 3, 3, 1, 1, 1, 2, 4, 32),
     ConvShape("res_stride2", 2, 15, 15, 128, 64, 3, 3, 2, 1, 1, 2, 4, 32),
     ConvShape("res_few_channels", 2, 32, 32, 3, 64, 7, 7, 2, 3, 1, 1, 1, 64),             # row-run kernel
-    ConvShape("res_long_k", 2, 14, 14, 256, 64, 3, 3, 1, 1, 1, 2, 4, 32),                 # split-K plans after tuning
+    ConvShape("res_long_k", 2, 14, 14, 256, 64, 3, 3, 1, 1, 1, 2, 4, 32),                 # split-K and balanced plans after tuning
+    ConvShape("res_pw_cout24", 2, 56, 56, 96, 24, 1, 1, 1, 0, 1, 2, 4, 8),                # pointwise, channels end inside a 32-block
+    ConvShape("res_pw_cin24_cout144", 1, 56, 56, 24, 144, 1, 1, 1, 0, 1, 2, 4, 16),
 ]
 
 
@@ -41,9 +43,9 @@ def test_residual_epilogue(nm, s, integer):
     xd, bd, rd = x.cuda(), b.cuda(), res.cuda()
     nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, True, kh=s.kh, kw=s.kw)    # reserves split-K scratch if any
     plans = _plans(nm, s)
-    for splits in (2, 3):
+    for splits, kblk in ((2, 0), (3, 0), (-1, 0), (-1, 2)):   # split-K, and balanced ranges (need the tuner's scratch)
         p = nm.nm_plan_t()
-        p.variant, p.bn, p.split = 4, 64, splits
+        p.variant, p.bn, p.split, p.kblk = 4, 64, splits, kblk
         plans.append(p)
     ran = set()
     for plan in plans:
