@@ -295,11 +295,27 @@ k_conv_rowrun(const ConvParams p, const RowCfg cfg, const __grid_constant__ CUte
                                ((static_cast<uint32_t>(lane >> 2) ^ static_cast<uint32_t>(bw)) << 4);
                 src += bw * (step8 >> 3);
                 uint32_t v[BM / 8];
+                // Rows 16 .. 95 lie inside every column's range of valid pixels on all but the border items
+                // (then for the whole warp): they are copied without the per-row test.
+                const bool inner = __all_sync(0xFFFFFFFFu, lo <= 16 && static_cast<uint32_t>(96 - lo) <= cnt);
+                if (inner) {
 #pragma unroll
-                for (int i = 0; i < BM / 8; ++i) {
-                    const bool valid = static_cast<uint32_t>(bw + i * 8 - lo) < cnt;
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(valid ? src : zero_row));
-                    src += step8;
+                    for (int i = 0; i < BM / 8; ++i) {
+                        if (i >= 2 && i < 12) {
+                            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(src));
+                        } else {
+                            const bool valid = static_cast<uint32_t>(bw + i * 8 - lo) < cnt;
+                            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(valid ? src : zero_row));
+                        }
+                        src += step8;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < BM / 8; ++i) {
+                        const bool valid = static_cast<uint32_t>(bw + i * 8 - lo) < cnt;
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(valid ? src : zero_row));
+                        src += step8;
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < BM / 8; ++i) {
