@@ -339,12 +339,12 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const int o0 = slice * cfg.bn;
             float bias_next = half < n_blk ? bias_lane_load(p.bias, o0 + half * 32, p.c_out, lane) : 0.f;   // first block's bias
             if (res_pass && half < n_blk) load_residual_box(rv, res_base + half * 32, p.c_out, res_rows, lane, cols_left - half * 32);
-            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
-            if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
-            if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
-            tc_fence_after();
-            // positions (of the equal ranges) that hold the rest of this item: first_pos + 1 .. last_pos
+            // positions (of the equal ranges) that hold the rest of this item: first_pos + 1 .. last_pos.  Their
+            // partial sums were stored long ago (they are those CTAs' first piece of work), so the flags are
+            // checked and, where no shortcut input occupies the registers, the first counterpart's sums of
+            // this warp's first block are requested BEFORE the wait for this CTA's own accumulator.
             uint32_t first_pos = 0, last_pos = 0;
+            bool ahead = false;
             if (finish) {
                 first_pos = gridDim.x - 1u - blockIdx.x;
                 const uint32_t u_last = (work + 1u) * static_cast<uint32_t>(n_sub) - 1u;
@@ -358,8 +358,18 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     for (uint32_t poll = 0; poll < kWaitPolls && !seen; ++poll) seen = ld_acquire_gpu(f) == 1u;
                     if (!seen) *abort_flag = 10;
                 }
-                if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
+                if (!res_pass && half < n_blk && !aborted(abort_flag)) {
+                    const float4* src = reinterpret_cast<const float4*>(slots + slot_floats * (gridDim.x - 2u - first_pos)) +
+                                        static_cast<size_t>(half) * 8 * BM + my_row;
+#pragma unroll
+                    for (int qq = 0; qq < 8; ++qq) rv[qq] = __ldcg(src + qq * BM);
+                    ahead = true;
+                }
             }
+            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
+            if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
+            if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
+            tc_fence_after();
             for (int blk = half; blk < n_blk; blk += 2, ++nb) {
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_addr + ab * cfg.bn + blk * 32, v);
@@ -382,7 +392,24 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     continue;
                 }
                 if (finish) {
-                    for (uint32_t pos = first_pos + 1u; pos <= last_pos; ++pos) {
+                    uint32_t pos_from = first_pos + 1u;
+                    if (ahead) {
+#pragma unroll
+                        for (int qq = 0; qq < 8; ++qq) {
+                            v[qq * 4 + 0] = __float_as_uint(__uint_as_float(v[qq * 4 + 0]) + rv[qq].x);
+                            v[qq * 4 + 1] = __float_as_uint(__uint_as_float(v[qq * 4 + 1]) + rv[qq].y);
+                            v[qq * 4 + 2] = __float_as_uint(__uint_as_float(v[qq * 4 + 2]) + rv[qq].z);
+                            v[qq * 4 + 3] = __float_as_uint(__uint_as_float(v[qq * 4 + 3]) + rv[qq].w);
+                        }
+                        if (blk + 2 < n_blk) {   // a block ahead
+                            const float4* nxt = reinterpret_cast<const float4*>(slots + slot_floats * (gridDim.x - 2u - first_pos)) +
+                                                static_cast<size_t>(blk + 2) * 8 * BM + my_row;
+#pragma unroll
+                            for (int qq = 0; qq < 8; ++qq) rv[qq] = __ldcg(nxt + qq * BM);
+                        }
+                        ++pos_from;
+                    }
+                    for (uint32_t pos = pos_from; pos <= last_pos; ++pos) {
                         const float4* src = reinterpret_cast<const float4*>(slots + slot_floats * (gridDim.x - 1u - pos)) +
                                             static_cast<size_t>(blk) * 8 * BM + my_row;
                         float4 t4[8];
