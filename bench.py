@@ -542,7 +542,8 @@ def main():
         traffic = recorded_traffic(dom, args.batch) if dom in KERNEL_SOURCE and not args.layer else None
         out["roofline"] = {
             "bound": "hbm", "achieved": dom_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": dom_gbs / pk["hbm_gbs"],
-            "traffic": traffic[0] / d["launches"] if traffic else None,
+            # per launch, averaged over the launches of the profiled step (its plans may differ by a layer or two)
+            "traffic": traffic[0] / float(traffic[1].get("launches_per_step", d["launches"])) if traffic else None,
             "peak_source": pk["source"] + " (burst copy figure)",
             "kernel": dom, "launches_per_step": d["launches"], "avg_launch_ms": d["ms"] / d["launches"],
             "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],
