@@ -599,18 +599,34 @@ def main():
                 nm.nm_conv2d(hnd, x_in, s.kh, s.kw, s.stride, s.pad, s.dil, bias, relu, y=y, plan=plan, residual=residual)
                 return y
 
+            branch = torch.cuda.Stream()          # a block's projection shortcut runs beside its main path
+            ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
+
             def chained_step(x_in=None, before_last=None):
+                main = torch.cuda.current_stream()
                 cur = conv(0, state[0][2] if x_in is None else x_in, True)
                 cur = nm.nm_maxpool2d(cur, 3, 2, 1, y=pool_out)
                 for pre in prefixes:
                     if before_last is not None and pre == prefixes[-1]:
                         before_last()    # the last block writes the step's output buffer
-                    shortcut = conv(idx[pre + "_ds"], cur, False) if pre + "_ds" in idx else cur
+                    forked = pre + "_ds" in idx
+                    if forked:
+                        ev_fork.record(main)
+                        branch.wait_event(ev_fork)
+                        with torch.cuda.stream(branch):
+                            shortcut = conv(idx[pre + "_ds"], cur, False)
+                            ev_join.record(branch)
+                    else:
+                        shortcut = cur
                     t = conv(idx[pre + "_c1"], cur, True)
                     if pre + "_c3" in idx:                       # bottleneck block
                         t = conv(idx[pre + "_c2"], t, True)
+                        if forked:
+                            main.wait_event(ev_join)
                         cur = conv(idx[pre + "_c3"], t, True, residual=shortcut)
                     else:                                        # basic block
+                        if forked:
+                            main.wait_event(ev_join)
                         cur = conv(idx[pre + "_c2"], t, True, residual=shortcut)
                 return cur
 
@@ -627,7 +643,8 @@ def main():
             out["chained"] = {"value": args.batch / (c_ms * 1e-3), "unit": UNIT, "ms_per_step": c_ms,
                               "finite": bool(torch.isfinite(last).all()),
                               "note": "conv backbone in dataflow order: stem, 3x3/2 max-pool, residual blocks with the "
-                                      "shortcut addition fused into the block's last convolution"}
+                                      "shortcut addition fused into the block's last convolution, projection "
+                                      "shortcuts on a second stream beside the block's main path"}
             # ... fed from the host: images copied in from pinned memory and the final feature map copied back,
             # every step, inside the timed region (what an inference loop around the backbone moves over PCIe)
             x0 = state[0][2]
