@@ -39,6 +39,19 @@ def test_binding_names_match_header(lib_path):
         assert hasattr(nm, name) or hasattr(nm._lib, name)
 
 
+def test_plan_struct_matches_the_header(lib_path):
+    """nm_plan_t is plain data that crosses the ABI: the binding's field order and size are the header's."""
+    from paper_2507_17301_b200 import nm
+    text = open(os.path.join(ROOT, "include", "nm.h")).read()
+    body = re.search(r"typedef struct \{([^}]*)\} nm_plan_t;", text).group(1)
+    fields = re.findall(r"int\s+(\w+)(?:\[(\d+)\])?;", body)
+    names = [n for n, _ in fields]
+    ints = sum(int(c) if c else 1 for _, c in fields)
+    assert names == [n for n, _ in nm.nm_plan_t._fields_]
+    assert ctypes.sizeof(nm.nm_plan_t) == 4 * ints == 64
+    assert [getattr(nm.nm_plan_t, n).offset for n in names[:5]] == [0, 4, 8, 12, 16]
+
+
 def test_argument_errors_without_gpu(lib_path):
     from paper_2507_17301_b200 import nm
     out = ctypes.c_void_p()
