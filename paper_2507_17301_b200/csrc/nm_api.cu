@@ -7,6 +7,8 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <mutex>
+#include <unordered_map>
 #include <vector>
 
 #include "nm_internal.h"
@@ -254,6 +256,21 @@ bool pdl_enabled()
     return on;
 }
 void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes)
+{
+    static std::mutex mu;
+    static std::unordered_map<uint64_t, size_t> in_force;   // (device, kernel) -> limit set so far
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const uint64_t key = (static_cast<uint64_t>(reinterpret_cast<uintptr_t>(kernel)) << 6) ^ static_cast<uint64_t>(dev & 63);
+    std::lock_guard<std::mutex> lock(mu);
+    const auto it = in_force.find(key);
+    if (it != in_force.end() && it->second >= bytes) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e == cudaSuccess) in_force[key] = bytes;
+    return e;
+}
 }  // namespace nmhost
 
 extern "C" {

@@ -651,7 +651,7 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     using Kernel = void (*)(const ConvParams, const ExpandCfg, const CUtensorMap, const CUtensorMap);
     const Kernel kernel = cfg.balanced ? (cfg.kblk == 2 ? k_conv_expand<2, true> : k_conv_expand<1, true>)
                                        : (cfg.kblk == 2 ? k_conv_expand<2, false> : k_conv_expand<1, false>);
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 4): %s", cudaGetErrorString(e));
     long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
     if (cfg.balanced) grid = sm_count();

@@ -371,7 +371,7 @@ nm_status_t launch_conv_pair(const ConvParams& p, const nm_plan_t* plan, cudaStr
     if (!nmtm::encode_x_im2col(p, BM, &tm_x) || !nmtm::encode_y_tiled(p, &tm_y))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 7)");
     const size_t smem = smem_bytes(cfg);
-    cudaError_t e = cudaFuncSetAttribute(k_conv_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_pair), smem);
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 7): %s", cudaGetErrorString(e));
     const int pairs_max = max_pairs(smem);   // every configuration takes a whole SM, so the first answer holds for all
     if (pairs_max < 1) return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: this device runs no clusters of two CTAs (variant 7)");

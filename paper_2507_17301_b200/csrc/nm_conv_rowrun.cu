@@ -418,7 +418,7 @@ nm_status_t launch_conv_rowrun(const ConvParams& p, const nm_plan_t* /*plan*/, c
         return fail(NM_ERR_UNSUPPORTED, "nm_conv2d: the row-run kernel does not take this layer");
     alignas(64) CUtensorMap tm_y;
     if (!encode_y_rows(p, &tm_y)) return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 5)");
-    cudaError_t e = cudaFuncSetAttribute(k_conv_rowrun, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_rowrun), smem);
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 5): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
     e = nmhost::launch_pdl(k_conv_rowrun, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_y);

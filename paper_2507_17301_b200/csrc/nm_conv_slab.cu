@@ -425,8 +425,7 @@ nm_status_t launch(const ConvParams& p, const SlabCfg& cfg, cudaStream_t st)
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: output tensor-map encoding failed");
     size_t smem = static_cast<size_t>(cfg.stages) * cfg.stage_bytes + 1024;
     if (smem < 78 * 1024) smem = 78 * 1024;  // never more than two CTAs (2 x 256 TMEM columns) per SM
-    cudaError_t e = cudaFuncSetAttribute(k_conv_slab<KC, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_slab<KC, TMA>), smem);
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 2): %s", cudaGetErrorString(e));
     const long long tiles_m = (p.pixels + BM - 1) / BM;
     const long long blocks = tiles_m * cfg.n_slices;

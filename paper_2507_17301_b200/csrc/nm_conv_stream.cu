@@ -502,8 +502,7 @@ nm_status_t launch(const ConvParams& p, const StreamCfg& cfg, cudaStream_t st)
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 3)");
     size_t smem = 1024 + static_cast<size_t>(cfg.stages) * cfg.stage_bytes + STAGING_BYTES;
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
-    cudaError_t e = cudaFuncSetAttribute(k_conv_stream<NK, MG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_stream<NK, MG>), smem);
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 3): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
     e = nmhost::launch_pdl(k_conv_stream<NK, MG>, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x, tm_w, tm_y);

@@ -391,7 +391,7 @@ nm_status_t launch_conv_window(const ConvParams& p, const nm_plan_t* plan, cudaS
     alignas(64) CUtensorMap tm_x;
     if (!encode_x_patch(p, cfg, &tm_x))
         return fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 6)");
-    cudaError_t e = cudaFuncSetAttribute(k_conv_window, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_window), smem);
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 6): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
     e = launch_pdl(k_conv_window, static_cast<unsigned>(grid), THREADS, smem, st, p, cfg, tm_x);

@@ -98,6 +98,10 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, 
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Raises a kernel's dynamic shared-memory limit on the current device, calling the runtime only when a launch
+// needs more than the limit already in force (the call would otherwise sit between every two launches).
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
+
 // Sets the calling thread's error text and returns `s`.
 nm_status_t fail(nm_status_t s, const char* fmt, ...);
 void count_launch(int n = 1);
