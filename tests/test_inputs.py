@@ -54,3 +54,28 @@ def test_mobilenet_v2_pointwise_shapes():
     macs = sum(s.ho * s.wo * s.c_in * s.c_out for s in layers)
     assert 250e6 < macs < 300e6
 
+
+
+def test_bench_host_logic(tmp_path, monkeypatch):
+    """bench.py's workload selection, algorithmic bytes and the look-up of recorded DRAM traffic (no GPU)."""
+    import bench
+
+    monkeypatch.setitem(bench.WORKLOAD, "net", "resnet")
+    r50 = bench.workload(64)
+    assert len(r50) == 53 and bench.workload_name(64) == "resnet50_conv_stack_b64_224_2of4"
+    stem = r50[0]
+    # stem: input 64 x 224 x 224 x 3, output 64 x 112 x 112 x 64, all 64 x 147 weights kept, one tile's indices, bias
+    assert bench.algorithmic_bytes(stem) == 4 * (64 * 224 * 224 * 3 + 64 * 112 * 112 * 64 + 64 * 147 + 64) + 2 * 147
+    assert bench.useful_flops(stem) == 2 * 64 * 112 * 112 * 64 * 147
+    monkeypatch.setitem(bench.WORKLOAD, "net", "mobilenet_v2")
+    assert len(bench.workload(8)) == 34 and bench.workload_name(8).startswith("mobilenet_v2_pointwise")
+    monkeypatch.setitem(bench.WORKLOAD, "net", "resnet")
+    # a traffic summary counts only while the kernel source it was taken from is unchanged
+    got = bench.recorded_traffic("k_conv_expand", 64)
+    if got is not None:
+        total, kv = got
+        assert total == float(kv["dram_bytes_per_step"]) and kv["source_sha256_16"] == bench.source_digest("k_conv_expand")
+        assert bench.recorded_traffic("k_conv_expand", 128)[0] == 2 * total
+    monkeypatch.setattr(bench, "source_digest", lambda kernel: "0" * 16)
+    assert bench.recorded_traffic("k_conv_expand", 64) is None
+    assert bench.recorded_traffic("k_no_such_kernel", 64) is None
