@@ -19,7 +19,8 @@
  *     (Algorithm 1, read with W[t, n] and C + t*V), i.e. the dense convolution
  *     with the pruned columns set to zero.
  *   Readings where the paper is silent: scores are summed in fp64 over the tile's
- *   rows in ascending row order; equal scores keep the lower column; a tail group of
+ *   rows in ascending row order; a score that is NaN ranks as +infinity; equal scores keep the
+ *   lower column; a tail group of
  *   m' < M columns keeps min(N, m'); a tail tile sums over the rows that exist;
  *   bias is added before an optional ReLU; out-of-range taps read zero.
  *
@@ -85,7 +86,9 @@ int nm_oracle_prune(const float* w, int c_out, int k, int n_keep, int m_group, i
             for (int i = 0; i < gsz; ++i) {
                 double s = 0.0;
                 for (int o = row0; o < row1; ++o) s += fabs((double)w[(size_t)o * k + g0 + i]);
-                score[i] = s;
+                /* a NaN score (a NaN weight) would make the comparisons below depend on position;
+                 * it ranks as +infinity, which keeps the order total (ties by column as usual) */
+                score[i] = isnan(s) ? (double)INFINITY : s;
                 keep[i] = 0;
             }
             /* retain the `take` largest; a later column wins only if strictly larger */

@@ -58,6 +58,30 @@ def test_hand_example_tail_group_and_tail_tile():
     assert oracle.kept_count(7, 2, 4) == 4
 
 
+def test_hand_example_non_finite_scores():
+    # The paper is silent on non-finite weights.  Reading: a NaN score ranks as +infinity (an
+    # infinite score already does), ties by column; a group still keeps exactly N columns.
+    nan, inf = float("nan"), float("inf")
+    w = np.array([[nan, 3, 2, 1, 1, nan, nan, 5]], dtype=np.float32)
+    _, indices = oracle.prune(w, 2, 4, 1)
+    assert indices.tolist() == [[0, 1, 5, 6]]          # NaN first or later in the group: kept either way
+    w = np.array([[1, 2, nan, 3, 7, -inf, 6, inf]], dtype=np.float32)
+    _, indices = oracle.prune(w, 1, 4, 1)
+    assert indices.tolist() == [[2, 5]]                # |-inf| = +inf ties with +inf: lower column
+    # a NaN in one row of a wider tile poisons that column's L1 sum only
+    w = np.array([[1, 9, 1, 1], [1, 1, nan, 1]], dtype=np.float32)
+    values, indices = oracle.prune(w, 1, 4, 2)
+    assert indices.tolist() == [[2]]
+    assert values[0].tolist() == [1.0] and np.isnan(values[1, 0])
+    # every (tile, group) still keeps exactly N
+    rng = _rng(11)
+    w = rng.standard_normal((8, 32)).astype(np.float32)
+    w[rng.integers(0, 8, 20), rng.integers(0, 32, 20)] = nan
+    _, indices = oracle.prune(w, 2, 4, 4)
+    assert indices.shape == (2, 16)
+    assert (indices // 4 == np.arange(16) // 2).all()
+
+
 # ---- sparsity identities printed in the paper ------------------------------------------------
 
 @pytest.mark.parametrize("n,m,sparsity", [(2, 4, 0.5), (3, 4, 0.25), (1, 4, 0.75), (4, 8, 0.5)])
