@@ -118,7 +118,9 @@ typedef struct {
  * `m_group` consecutive columns the `n_keep` highest-scoring units are RETAINED (N counts kept
  * columns, N = (1 - sparsity) * M) and all rows of the tile share that kept set.
  * Deterministic rules where the paper is silent: scores are fp64 sums over the tile's rows in
- * ascending row order; of two equal scores the lower column is kept; a tail group of m' < M
+ * ascending row order; a score that is NaN (a NaN weight in the column) ranks as +infinity, like the
+ * score of a column holding an infinite weight, so the order of the scores is total for every input
+ * and every group keeps exactly N columns; of two equal scores the lower column is kept; a tail group of m' < M
  * columns keeps min(N, m'); a tail tile (c_out % tile_t rows) scores over the rows it has.
  *
  *   w_dense   device, fp32 [c_out][kh][kw][c_in]; read only, may be freed after the stream
@@ -149,7 +151,15 @@ nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, 
  * NM_ERR_UNSUPPORTED and does nothing.  All calls share the one scratch array: calls whose kernels
  * could overlap on the GPU (other streams or threads) race, so issue them one after another on one
  * stream.  The first call on a given device looks up the array's device address (once per device,
- * cached); make that first call outside any stream capture.  Asynchronous on `cuda_stream`.
+ * cached); make that first call outside any stream capture.  With lazy module loading (the CUDA
+ * default) that first call is also when the runtime loads the module holding the array: the 4.5 MiB
+ * are reserved on the device then, and the load may synchronise it.  So "allocates nothing" holds
+ * from the second call on: make one warm-up call per device at start-up, while memory is still to
+ * be had.  The cached address does not survive a cudaDeviceReset.  Same limits as nm_prune
+ * (kh, kw <= 255, tile_t <= 256), so that the result can be fed to nm_weights_import; `values` and
+ * `indices` must hold c_out * kk floats and ceil(c_out / tile_t) * kk uint16 (not checked here; the
+ * Python binding checks its tensors).  No column is ever placed outside a group's N slots, whatever
+ * the weights hold (NaN and infinities included).  Asynchronous on `cuda_stream`.
  */
 #define NM_NOALLOC_MAX_CELLS (1 << 19)
 nm_status_t nm_prune_noalloc(const float* w_dense, int c_out, int kh, int kw, int c_in, int n_keep,
@@ -180,9 +190,10 @@ nm_status_t nm_weights_export(const nm_weights_t* w, float* values, uint16_t* in
 
 /*
  * Builds a handle from an already compressed model (the inverse of nm_weights_export; this is the
- * checkpoint path).  Validates on the device that every index row is strictly ascending and
- * < K; the group structure is not re-checked.  Same errors as nm_prune, plus INVALID_ARG for a bad
- * index row (detected synchronously).
+ * checkpoint path).  Validates on the device that every index row is strictly ascending, < K, and
+ * holds the N:M structure the kernels rely on (retained column j lies in group j / N of M
+ * consecutive columns).  Same errors as nm_prune, plus INVALID_ARG for a bad index row (detected
+ * synchronously).
  */
 nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int c_out, int kh,
                               int kw, int c_in, int n_keep, int m_group, int tile_t,

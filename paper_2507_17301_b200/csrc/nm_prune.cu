@@ -2,7 +2,8 @@
 // kernel-side copies of the compressed form (Sec. 2.1; inputs W and Idx of Algorithm 1).
 //
 // Four small kernels, all one thread per (tile, column) or (row, retained column):
-//   score    s[r][k]   = sum over the tile's rows of |w[o][k]|, fp64, ascending row order
+//   score    s[r][k]   = sum over the tile's rows of |w[o][k]|, fp64, ascending row order; a sum that
+//            is NaN (a NaN weight) counts as +infinity, so that the order below is total
 //   select   keep[r][k] = 1 iff fewer than N columns of k's group beat it, where column i beats
 //            column k when s[i] > s[k], or s[i] == s[k] and i < k (lower column wins ties)
 //   compact  position of each kept column = N * group + number of kept columns before it in its
@@ -27,7 +28,9 @@ __global__ void k_score(const float* __restrict__ w, int c_out, int k, int tile_
     const int row1 = min(row0 + tile_t, c_out);
     double s = 0.0;
     for (int o = row0; o < row1; ++o) s += fabs(static_cast<double>(w[static_cast<size_t>(o) * k + col]));
-    score[static_cast<size_t>(r) * k + col] = s;
+    // NaN compares false with everything: such a column would neither beat nor be beaten, and its
+    // group would keep more than N columns.  It ranks as +infinity instead (ties by column).
+    score[static_cast<size_t>(r) * k + col] = (s == s) ? s : static_cast<double>(INFINITY);
 }
 
 __global__ void k_select(const double* __restrict__ score, int k, int n_keep, int m_group,
@@ -80,6 +83,9 @@ __global__ void k_compact(const uint8_t* __restrict__ keep, int k, int kk, int k
     const int g = col / m_group;
     int pos = g * n_keep;  // every earlier group is a full one and kept exactly n_keep
     for (int i = g * m_group; i < col; ++i) pos += kp[i];
+    // a group never holds more than N kept columns (the order of the scores is total); the bound
+    // makes sure that no input whatsoever can place a column outside its group's slots
+    if (pos >= min(kk, (g + 1) * n_keep)) return;
     indices[static_cast<size_t>(r) * kk + pos] = static_cast<uint16_t>(col);
     const int c = col % c_in, tap = col / c_in;
     taps[static_cast<size_t>(r) * kk_pad + pos] =
@@ -157,14 +163,18 @@ __global__ void k_expand(const float* __restrict__ values, const uint16_t* __res
         nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
 }
 
-// Import path: every index row must be strictly ascending and below k.
-__global__ void k_check_indices(const uint16_t* __restrict__ indices, int kk, int k, int* __restrict__ bad)
+// Import path: every index row must be strictly ascending and below k, and hold the N:M structure
+// the kernels rely on: retained column j lies in group j / N (a tail group of m' < M columns keeps
+// min(N, m'), which the same quotient covers).
+__global__ void k_check_indices(const uint16_t* __restrict__ indices, int kk, int k, int n_keep, int m_group,
+                                int* __restrict__ bad)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     const int r = blockIdx.y;
     if (j >= kk) return;
     const int v = indices[static_cast<size_t>(r) * kk + j];
-    if (v >= k || (j > 0 && indices[static_cast<size_t>(r) * kk + j - 1] >= v)) atomicExch(bad, 1);
+    if (v >= k || (j > 0 && indices[static_cast<size_t>(r) * kk + j - 1] >= v) || v / m_group != j / n_keep)
+        atomicExch(bad, 1);
 }
 
 #define NM_CUDA_TRY(call)                                                                                   \
@@ -298,7 +308,7 @@ nm_status_t build_from_compressed(const float* values, const uint16_t* indices, 
     NM_CUDA_TRY(cudaMemsetAsync(h->taps, 0xFF, static_cast<size_t>(h->n_tiles) * h->kk_pad * sizeof(uint32_t), st));
     NM_CUDA_TRY(cudaMemsetAsync(h->status + 3, 0, sizeof(int), st));
     if (h->kk > 0) {
-        k_check_indices<<<grid_idx, blk, 0, st>>>(h->indices, h->kk, h->k, h->status + 3);
+        k_check_indices<<<grid_idx, blk, 0, st>>>(h->indices, h->kk, h->k, h->n_keep, h->m_group, h->status + 3);
         k_taps_from_indices<<<grid_idx, blk, 0, st>>>(h->indices, h->kk, h->kk_pad, h->c_in, h->kw, h->taps);
         count_launch(2);
     }
@@ -307,7 +317,7 @@ nm_status_t build_from_compressed(const float* values, const uint16_t* indices, 
     NM_CUDA_TRY(cudaGetLastError());
     NM_CUDA_TRY(cudaMemcpyAsync(&bad, h->status + 3, sizeof(int), cudaMemcpyDeviceToHost, st));
     NM_CUDA_TRY(cudaStreamSynchronize(st));
-    if (bad) st_out = fail(NM_ERR_INVALID_ARG, "nm_weights_import: an index row is not strictly ascending below K");
+    if (bad) st_out = fail(NM_ERR_INVALID_ARG, "nm_weights_import: an index row is not strictly ascending below K, or does not hold N columns per group of M");
 done:
     return st_out;
 }

@@ -19,7 +19,10 @@
 // The array's name is only a host-side handle in host code; the device address is looked up once
 // per device with cudaGetSymbolAddress while that device is current and cached.  That lookup
 // happens on the first call for a device, which should therefore be made outside any stream
-// capture.
+// capture.  With lazy module loading that first call is also the moment the CUDA runtime loads the
+// module holding the array, i.e. when the 4.5 MiB are actually reserved on the device (and the
+// load may synchronise): "allocates nothing" holds from the second call on, so make one warm-up
+// call per device at start-up.  The cached address does not survive a cudaDeviceReset.
 #include <mutex>
 
 #include "nm_internal.h"
@@ -54,7 +57,8 @@ nm_status_t scratch_for_current_device(unsigned char** out)
 }
 
 // The same three steps as the allocating pruner (Sec. 3.1), restated here so that this entry
-// point shares no code path with it: L1 score per (tile, column) in fp64 over ascending rows;
+// point shares no code path with it: L1 score per (tile, column) in fp64 over ascending rows (a NaN
+// sum ranks as +infinity);
 // keep a column iff fewer than N columns of its group beat it (greater score, or equal score and
 // lower position); place each kept column at N * group + kept-before-it.
 __global__ void k_static_score(const float* __restrict__ w, int c_out, int k, int tile_t, double* __restrict__ score)
@@ -65,7 +69,7 @@ __global__ void k_static_score(const float* __restrict__ w, int c_out, int k, in
     const int row0 = r * tile_t, row1 = min(row0 + tile_t, c_out);
     double s = 0.0;
     for (int o = row0; o < row1; ++o) s += fabs(static_cast<double>(w[static_cast<size_t>(o) * k + col]));
-    score[static_cast<size_t>(r) * k + col] = s;
+    score[static_cast<size_t>(r) * k + col] = (s == s) ? s : static_cast<double>(INFINITY);   // NaN ranks as +infinity
 }
 
 __global__ void k_static_select(const double* __restrict__ score, int k, int n_keep, int m_group,
@@ -93,6 +97,7 @@ __global__ void k_static_place(const unsigned char* __restrict__ keep, int k, in
     const int g = col / m_group;
     int pos = g * n_keep;
     for (int i = g * m_group; i < col; ++i) pos += kp[i];
+    if (pos >= min(kk, (g + 1) * n_keep)) return;   // never outside the group's slots, whatever the input
     indices[static_cast<size_t>(r) * kk + pos] = static_cast<uint16_t>(col);
 }
 
@@ -117,6 +122,9 @@ extern "C" nm_status_t nm_prune_noalloc(const float* w_dense, int c_out, int kh,
     if (n_keep < 1 || m_group < 1 || n_keep > m_group)
         return nmhost::fail(NM_ERR_INVALID_ARG, "nm_prune_noalloc: need 1 <= n_keep <= m_group (got %d:%d)", n_keep, m_group);
     if (tile_t < 1) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_prune_noalloc: tile_t must be >= 1");
+    // the limits of nm_prune / nm_weights_import, so that whatever this call produces can be imported
+    if (kh > 255 || kw > 255) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_prune_noalloc: kernel extent above 255");
+    if (tile_t > 256) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_prune_noalloc: tile_t above 256");
     const long long k = static_cast<long long>(kh) * kw * c_in;
     if (k > 65535) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_prune_noalloc: K = %lld exceeds the uint16 index range", k);
     if (c_out > 65535) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_prune_noalloc: c_out above 65535");

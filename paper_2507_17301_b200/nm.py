@@ -175,6 +175,13 @@ def nm_prune_noalloc(w_dense: torch.Tensor, n_keep: int, m_group: int, tile_t: i
     vptr = _dev_f32(values, "values")
     if not (indices.is_cuda and indices.dtype == torch.uint16 and indices.is_contiguous()):
         raise TypeError("indices must be a contiguous uint16 CUDA tensor")
+    if n_keep >= 1 and m_group >= n_keep and tile_t >= 1:   # otherwise the library reports the bad argument
+        k = kh * kw * c_in
+        kk = (k // m_group) * n_keep + min(k % m_group, n_keep)
+        n_tiles = -(-c_out // tile_t)
+        if values.numel() < c_out * kk or indices.numel() < n_tiles * kk:
+            raise TypeError(f"values needs {c_out * kk} elements and indices {n_tiles * kk} "
+                            f"(got {values.numel()} and {indices.numel()})")
     _check(_lib.nm_prune_noalloc(ptr, c_out, kh, kw, c_in, n_keep, m_group, tile_t, vptr, indices.data_ptr(),
                                  _stream()))
 

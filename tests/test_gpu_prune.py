@@ -63,6 +63,40 @@ def test_ties_resolve_like_the_oracle(nm):
     _check(nm, torch.zeros(16, 1, 1, 32), 2, 4, 8)
 
 
+def test_non_finite_weights_keep_n_per_group_and_match_the_oracle(nm):
+    # a NaN score ranks as +infinity on both sides; no group keeps more than N, so nothing is
+    # placed outside the index array (the placement is bounded as well)
+    g = torch.Generator().manual_seed(9)
+    w = torch.randn((40, 3, 3, 8), generator=g)
+    flat = w.view(-1)
+    pick = torch.randperm(flat.numel(), generator=g)[:60]
+    flat[pick[:30]] = float("nan")
+    flat[pick[30:45]] = float("inf")
+    flat[pick[45:]] = float("-inf")
+    w[39, 2, 2, 4:] = float("nan")                      # the last group of the last tile, whole
+    for n, m, t in ((2, 4, 8), (1, 4, 16), (3, 8, 1), (2, 4, 64)):
+        hnd = nm.nm_prune(w.cuda(), n, m, t)
+        v, i = nm.nm_weights_export(hnd)
+        torch.cuda.synchronize()
+        vr, ir = oracle.prune(w.numpy(), n, m, t)
+        assert np.array_equal(i.cpu().numpy(), ir)
+        assert np.array_equal(v.cpu().numpy().view(np.uint32), vr.view(np.uint32))
+        assert (ir.astype(np.int64) // m == np.arange(ir.shape[1]) // n).all()
+
+
+def test_import_refuses_rows_without_the_group_structure(nm):
+    # strictly ascending and below K, but three columns of the first group and one of the second
+    s = inputs.config_tiny()
+    hnd = nm.nm_prune(inputs.make_weights(s).cuda(), 2, 4, 8)
+    v, i = nm.nm_weights_export(hnd)
+    bad = i.cpu().view(torch.int16).clone()
+    bad[1, 0:4] = torch.tensor([0, 1, 2, 5], dtype=torch.int16)
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_weights_import(v, bad.view(torch.uint16).cuda(), 3, 3, 16, 2, 4, 8)
+    assert e.value.status == nm.NM_ERR_INVALID_ARG
+    assert "group" in str(e.value)
+
+
 def test_import_round_trip_and_validation(nm):
     s = inputs.config_tiny()
     w = inputs.make_weights(s)
