@@ -80,7 +80,17 @@ typedef struct nm_weights nm_weights_t;
  *                staging its own 128 pixels and half of the weight rows of a 256 x bn MMA, which
  *                halves the shared-memory traffic per FLOP on reduction-heavy layers (needs the
  *                conditions of variant 4, bn 128 or 256, c_out % bn == 0).
- *   bn       output channels per CTA / work item (variants 2, 3: a multiple of tile_t; variant 4: a
+ *            8 = select kernel (persistent; contracts over the retained columns only: the dense
+ *                activations of a chunk are staged once per CTA, each thread reads its pixel's row with
+ *                16-byte loads and picks every tile's retained columns with M - N bitwise selects per
+ *                column under precomputed masks; one MMA issuer thread per tile; needs N:M one of
+ *                1:4 2:4 3:4 1:8 2:8 4:8, K % M == 0, c_in a multiple of the chunk's 64 (3:4: 32) source
+ *                columns, tile_t % 16 == 0, c_out % tile_t == 0, an input of at least 128 KiB).  Activation
+ *                loads (`loads`): im2col-mode TMA loads (any stride / dilation), or, for stride-1 layers
+ *                whose output has the input's size, "patch" loads that fetch a pixel block and its halo
+ *                once for all kh * kw taps.  `stages` = activation ring depth; `ksplit` > 1 splits the
+ *                reduction axis like variant 4's split (same scratch, same second pass).
+ *   bn       output channels per CTA / work item (variants 2, 3, 8: a multiple of tile_t; variant 4: a
  *            multiple of 32 up to 256 that divides c_out rounded up to a multiple of 32; variant 6: a multiple
  *            of 32 up to 256 that divides c_out; variant 7: 128 or 256), 0 = default
  *   stages   depth of the shared-memory ring, 0 = default
@@ -104,7 +114,10 @@ typedef struct {
     int stages;
     int split;
     int kblk;
-    int reserved[11];
+    int loads;    /* variant 8: 0 = the library's choice, 1 = im2col loads, 2 = patch loads */
+    int issuers;  /* variant 8: MMA issuer threads, 1 .. tiles per work item (0 = one per tile) */
+    int ksplit;   /* variant 8: ranges the reduction axis is split into, 1-8 (0 = 1); more than one needs scratch */
+    int reserved[8];
 } nm_plan_t;
 
 /* ---------------------------------------------------------------------------------------------

@@ -36,6 +36,8 @@ void free_handle_memory(nm_weights* h)
     cudaFree(h->wt2);
     cudaFree(h->rel2);
     cudaFree(h->wx);
+    cudaFree(h->w3);
+    cudaFree(h->sel3);
     cudaFree(h->splitk);
     h->magic = 0;
     delete h;
@@ -128,6 +130,9 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     p->wx_rows = w->wx_rows;
     p->splitk = w->splitk;
     p->splitk_bytes = w->splitk_bytes;
+    p->w3 = w->w3;
+    p->sel3 = w->sel3;
+    p->sel_s = w->sel_s; p->sel_kc = w->sel_kc; p->sel_mw = w->sel_mw;
     return NM_OK;
 }
 
@@ -154,6 +159,8 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
             return nmhost::launch_conv_window(p, plan, st);
         case 7:
             return nmhost::launch_conv_pair(p, plan, st);
+        case 8:
+            return nmhost::launch_conv_select(p, plan, st);
         default:
             return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
     }
@@ -164,6 +171,16 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
 {
     std::vector<nm_plan_t> out;
     nm_plan_t a;
+    std::memset(&a, 0, sizeof(a));
+    // select kernel (contracts over the retained columns only): all of a tile group's channels per CTA down to one
+    // tile, with the activation loads it prefers for the shape, and with the reduction axis split where few work
+    // items exist (the split plans need the handle's scratch)
+    for (int ksplit : {1, 2, 3, 4}) {
+        for (int bn : {256, 128, 64}) {
+            a.variant = 8; a.bn = bn; a.ksplit = ksplit;
+            if (bn % p.tile_t == 0 && nmhost::select_plan_ok(p, &a)) out.push_back(a);
+        }
+    }
     std::memset(&a, 0, sizeof(a));
     for (int mt : {2, 3, 4, 1}) {           // window kernel (stride-1 spatial kernels)
         for (int bn : {64, 128, 256}) {
@@ -230,7 +247,7 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     if (const char* allow = std::getenv("NM_AUTOTUNE_VARIANTS")) {
         std::vector<nm_plan_t> kept;
         for (const nm_plan_t& c : out)
-            if (std::strchr(allow, '0' + c.variant)) kept.push_back(c);
+            if (c.variant < 10 && std::strchr(allow, '0' + c.variant)) kept.push_back(c);
         if (!kept.empty()) out.swap(kept);
     }
     return out;
@@ -285,6 +302,7 @@ nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, 
     s = nmhost::prune_on_device(w_dense, h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_expanded_layout(h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_select_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         return s;
@@ -303,6 +321,7 @@ nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int 
     s = nmhost::build_from_compressed(values, indices, h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_expanded_layout(h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_select_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         *out = nullptr;
@@ -360,6 +379,7 @@ nm_status_t nm_plan_scratch_bytes(const nm_weights_t* w, int batch, int h, int w
     if (s != NM_OK) return s;
     if (plan && plan->variant == 4 && plan->split > 1) *bytes = nmhost::expand_splitk_bytes(p, plan->split);
     if (plan && plan->variant == 4 && plan->split == -1) *bytes = nmhost::expand_balanced_bytes(plan->bn > 0 ? plan->bn : 256);
+    if (plan && plan->variant == 8 && plan->ksplit > 1) *bytes = nmhost::select_splitk_bytes(p, plan->ksplit);
     return NM_OK;
 }
 
@@ -485,7 +505,7 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         const long long pix_blocks = (p.pixels + 127) / 128;
         const bool few_items = pix_blocks * ((p.c_out + 255) / 256) < n_sm && p.k / 32 >= 32;
-        size_t need = few_items && p.wx ? nmhost::expand_splitk_bytes(p, 4) : 0;
+        size_t need = few_items && (p.wx || p.w3) ? nmhost::expand_splitk_bytes(p, 4) : 0;
         // ... and layers with fewer than three rounds of work items with (item, stage) ranges balanced over the SMs
         const bool uneven = pix_blocks * ((p.c_out + 255) / 256) < 3ll * n_sm;
         if (uneven && p.wx && nmhost::expand_balanced_bytes(256) > need) need = nmhost::expand_balanced_bytes(256);

@@ -660,19 +660,23 @@ nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaS
     nmhost::count_launch(1);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (variant 4): %s", cudaGetErrorString(e));
-    if (cfg.ksplit > 1) {
-        const size_t n4 = static_cast<size_t>(p.pixels) * p.c_out / 4;
-        const size_t stride4 = static_cast<size_t>(cfg.p_pad) * p.c_out / 4;
-        size_t blocks = (n4 + 255) / 256;
-        if (blocks > static_cast<size_t>(sm_count()) * 8) blocks = static_cast<size_t>(sm_count()) * 8;
-        e = nmhost::launch_pdl(k_splitk_reduce, static_cast<unsigned>(blocks), 256u, 0, st,
-                               reinterpret_cast<const float4*>(p.splitk), cfg.ksplit, stride4, n4, p.c_out / 4,
-                               reinterpret_cast<const float4*>(p.bias), reinterpret_cast<const float4*>(p.residual), p.relu,
-                               reinterpret_cast<float4*>(p.y));
-        nmhost::count_launch(1);
-        if (e == cudaSuccess) e = cudaGetLastError();
-        if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (split-K reduction): %s", cudaGetErrorString(e));
-    }
+    if (cfg.ksplit > 1) return launch_splitk_reduce(p, cfg.ksplit, cfg.p_pad, st);
+    return NM_OK;
+}
+
+nm_status_t launch_splitk_reduce(const ConvParams& p, int splits, int p_pad, cudaStream_t st)
+{
+    const size_t n4 = static_cast<size_t>(p.pixels) * p.c_out / 4;
+    const size_t stride4 = static_cast<size_t>(p_pad) * p.c_out / 4;
+    size_t blocks = (n4 + 255) / 256;
+    if (blocks > static_cast<size_t>(sm_count()) * 8) blocks = static_cast<size_t>(sm_count()) * 8;
+    cudaError_t e = nmhost::launch_pdl(k_splitk_reduce, static_cast<unsigned>(blocks), 256u, 0, st,
+                                       reinterpret_cast<const float4*>(p.splitk), splits, stride4, n4, p.c_out / 4,
+                                       reinterpret_cast<const float4*>(p.bias), reinterpret_cast<const float4*>(p.residual),
+                                       p.relu, reinterpret_cast<float4*>(p.y));
+    nmhost::count_launch(1);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(NM_ERR_CUDA, "nm_conv2d launch (split-K reduction): %s", cudaGetErrorString(e));
     return NM_OK;
 }
 

@@ -33,6 +33,11 @@ struct nm_weights {
     size_t splitk_bytes;
     float* wx;           // [ceil(k / 32)][wx_rows][32] TF32, rows swizzled (see k_expand); NULL when the shape rules the variant out
     int wx_rows;         // c_out rounded up to a multiple of 32 (the rows past c_out are zero)
+    // Select layout (variant 8): chunks of sel_s source columns of which every tile keeps sel_kc; NULL when the
+    // pattern or the shape rules the variant out.
+    float* w3;           // [k / sel_s][c_out][32] TF32, rows swizzled (see k_build_w3)
+    uint32_t* sel3;      // [k / sel_s][n_tiles][sel_mw] select masks (see k_build_sel3)
+    int sel_s, sel_kc, sel_mw;
 };
 
 // Geometry handed to the convolution kernels.
@@ -58,9 +63,13 @@ struct ConvParams {
     // expanded layout (variant 4)
     const float* wx;
     int wx_rows;
-    // split-K scratch of the handle (variant 4 with plan.split > 1)
+    // split-K scratch of the handle (variant 4 with plan.split > 1, variant 8 with plan.ksplit > 1)
     float* splitk;
     size_t splitk_bytes;
+    // select layout (variant 8)
+    const float* w3;
+    const uint32_t* sel3;
+    int sel_s, sel_kc, sel_mw;
 };
 
 #ifdef __CUDACC__
@@ -126,6 +135,10 @@ size_t expand_splitk_bytes(const ConvParams& p, int splits);   // scratch a spli
 size_t expand_balanced_bytes(int bn);                          // scratch a balanced plan (split = -1) with this bn needs
 nm_status_t launch_conv_expand(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 
+// second pass of a plan that splits the reduction axis: y = act(sum of the `splits` partial sums
+// [split][p_pad pixels][c_out] in p.splitk + bias + shortcut)
+nm_status_t launch_splitk_reduce(const ConvParams& p, int splits, int p_pad, cudaStream_t st);
+
 // nm_conv_rowrun.cu — variant 5
 bool rowrun_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_rowrun(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
@@ -141,4 +154,10 @@ nm_status_t launch_conv_pair(const ConvParams& p, const nm_plan_t* plan, cudaStr
 // nm_conv_stream.cu — variant 3
 bool stream_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 nm_status_t launch_conv_stream(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
+// nm_conv_select.cu — variant 8
+nm_status_t build_select_layout(nm_weights* h, cudaStream_t st);
+bool select_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+size_t select_splitk_bytes(const ConvParams& p, int splits);
+nm_status_t launch_conv_select(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 }  // namespace nmhost

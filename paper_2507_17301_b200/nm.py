@@ -32,11 +32,12 @@ class NmError(RuntimeError):
 
 class nm_plan_t(ctypes.Structure):
     _fields_ = [("variant", ctypes.c_int), ("bn", ctypes.c_int), ("stages", ctypes.c_int),
-                ("split", ctypes.c_int), ("kblk", ctypes.c_int), ("reserved", ctypes.c_int * 11)]
+                ("split", ctypes.c_int), ("kblk", ctypes.c_int), ("loads", ctypes.c_int),
+                ("issuers", ctypes.c_int), ("ksplit", ctypes.c_int), ("reserved", ctypes.c_int * 8)]
 
     def as_dict(self):
         return {"variant": self.variant, "bn": self.bn, "stages": self.stages, "split": self.split,
-                "kblk": self.kblk}
+                "kblk": self.kblk, "loads": self.loads, "issuers": self.issuers, "ksplit": self.ksplit}
 
 
 def _load():
