@@ -83,7 +83,7 @@ typedef struct nm_weights nm_weights_t;
  *            8 = select kernel (persistent; contracts over the retained columns only: the dense
  *                activations of a chunk are staged once per CTA, each thread reads its pixel's row with
  *                16-byte loads and picks every tile's retained columns with M - N bitwise selects per
- *                column under precomputed masks; one MMA issuer thread per tile; needs N:M one of
+ *                column under precomputed masks; up to four MMA issuer threads; needs N:M one of
  *                1:4 2:4 3:4 1:8 2:8 4:8, K % M == 0, c_in a multiple of the chunk's 64 (3:4: 32) source
  *                columns, tile_t % 16 == 0, c_out % tile_t == 0, an input of at least 128 KiB).  Activation
  *                loads (`loads`): im2col-mode TMA loads (any stride / dilation), or, for stride-1 layers
@@ -115,7 +115,7 @@ typedef struct {
     int split;
     int kblk;
     int loads;    /* variant 8: 0 = the library's choice, 1 = im2col loads, 2 = patch loads */
-    int issuers;  /* variant 8: MMA issuer threads, 1 .. tiles per work item (0 = one per tile) */
+    int issuers;  /* variant 8: MMA issuer threads, 1-4 and at most the work item's MMA units (0 = as many as possible) */
     int ksplit;   /* variant 8: ranges the reduction axis is split into, 1-8 (0 = 1); more than one needs scratch */
     int reserved[8];
 } nm_plan_t;

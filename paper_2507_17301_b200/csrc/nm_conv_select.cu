@@ -19,17 +19,20 @@
 //                         a ninth of the im2col form's bytes through the TMA unit.
 //   weight producer       one bulk copy per chunk brings the G tiles' retained weights [G*T x KC]
 //   (1 thread)            (stored as the swizzled shared-memory image), another their select masks.
-//   compactors (8 warps)  thread = pixel row = TMEM lane, two warps per lane quadrant (one per half of
-//                         the chunk).  Each reads its row's share of the chunk ONCE with conflict-free
-//                         16-byte loads and, for every tile of the item, picks that tile's retained
-//                         columns out of its registers: the j-th retained column of a group of M lies
-//                         at one of the positions j .. j + (M - N), so it is a chain of M - N bitwise
-//                         selects (lop3) under warp-uniform masks precomputed at pruning time.  The
-//                         result goes to the tile's operand columns in tensor memory (tcgen05.st).
-//   MMA issuers           D[128 x T] += A[tmem] * W[smem]^T, KC / 8 tcgen05.mma per tile and chunk
-//   (1 thread per tile,   (the T accumulators of Algorithm 1 are T TMEM columns).  A lone thread issues
-//   up to 4)              an MMA every ~125 cycles whatever its size, and a 128 x 64 x 8 MMA runs in a
-//                         quarter of that: each tile of an item therefore has its own issuer thread.
+//   compactors (2 teams   thread = pixel row = TMEM lane, one warp per lane quadrant and team; the teams take
+//   of 4 warps)           alternate chunks, so that the barrier round trips and load latencies of one chunk
+//                         overlap the selects of the other.  A thread reads its row of the chunk ONCE with
+//                         conflict-free 16-byte loads (half a chunk at a time) and, for every tile of the
+//                         item, picks that tile's retained columns out of its registers: the j-th retained
+//                         column of a group of M lies at one of the positions j .. j + (M - N), so it is a
+//                         chain of M - N bitwise selects (lop3) under warp-uniform masks precomputed at
+//                         pruning time.  The result goes to the tile's operand columns in tensor memory
+//                         (tcgen05.st).
+//   MMA issuers           D[128 x n] += A[tmem] * W[smem]^T, KC / 8 tcgen05.mma per chunk and unit, a unit
+//   (up to 4 threads)     being n = BN / 4 accumulator columns of one tile (the T accumulators of Algorithm 1
+//                         are T TMEM columns).  A lone thread issues an MMA every ~125 cycles whatever its
+//                         size, a 128 x 64 x 8 MMA runs in 35: the units of an item are dealt to up to four
+//                         issuer threads, each with accumulator columns of its own.
 //   epilogue (4 warps)    TMEM -> registers, + bias, (+ shortcut), ReLU, staged through shared memory
 //                         and written to NHWC with TMA stores; with two accumulator buffers it
 //                         overlaps the next item's main loop.
@@ -57,6 +60,7 @@ constexpr int STAGING_BYTES = 4 * 2 * 4096;
 
 struct SelCfg {
     int g, bn, n_slices, n_acc, n_iss;
+    int mma_n, n_units; // accumulator columns per MMA and MMA units per work item (bn = n_units * mma_n)
     int patch;          // 1 = patch loads, 0 = im2col loads
     int taps;           // chunks per activation stage: kh * kw (patch) or 1 (im2col)
     int n_cb;           // chunks per tap = c_in / S
@@ -74,6 +78,18 @@ struct SelCfg {
 };
 
 __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
+
+// Bounded wait that also gives up once another role has raised the abort flag (looked at every 64 polls, off
+// the path of a wait that is already satisfied).
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* flag)
+{
+    if (mbar_test_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < kWaitPolls; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *flag != 0) return false;
+    }
+    return false;
+}
 
 // Four consecutive 32-bit words of shared memory into dst[0..3].
 __device__ __forceinline__ void lds128(uint32_t addr, uint32_t* dst)
@@ -143,7 +159,6 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
     __shared__ uint64_t s_pfull[MAX_P], s_pfree[MAX_P], s_wfull[MAX_W], s_wfree[MAX_W], s_aready[MAX_SETS],
         s_afree[MAX_SETS], s_accfull[2], s_accfree[2];
     __shared__ __align__(128) float s_zero[32];
-    __shared__ int s_shift[MAX_TAPS];
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
 
@@ -161,14 +176,14 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
     if (tid == 0) {
         for (int i = 0; i < MAX_P; ++i) {
             mbar_init(smem_u32(&s_pfull[i]), 1);              // producer's expect-tx arrival
-            mbar_init(smem_u32(&s_pfree[i]), 8);              // compactor warps
+            mbar_init(smem_u32(&s_pfree[i]), cfg.taps > 1 ? 8 : 4);   // compactor warps that read the stage
         }
         for (int i = 0; i < MAX_W; ++i) {
             mbar_init(smem_u32(&s_wfull[i]), 1);
-            mbar_init(smem_u32(&s_wfree[i]), 8 + cfg.n_iss);  // compactor warps (masks) + MMA commits (weights)
+            mbar_init(smem_u32(&s_wfree[i]), 4 + cfg.n_iss);  // one compactor team (masks) + MMA commits (weights)
         }
         for (int i = 0; i < MAX_SETS; ++i) {
-            mbar_init(smem_u32(&s_aready[i]), 8);             // compactor warps
+            mbar_init(smem_u32(&s_aready[i]), 4);             // one compactor team
             mbar_init(smem_u32(&s_afree[i]), cfg.n_iss);      // MMA commits
         }
         for (int i = 0; i < 2; ++i) {
@@ -181,12 +196,6 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         tma_prefetch_desc(&tm_y);
     }
     if (tid < 32) s_zero[tid] = 0.f;
-    if (tid >= 32 && tid < 32 + MAX_TAPS) {
-        // patch form: rows between the first patch row and a pixel's source row of tap (i, j)
-        const int t = tid - 32;
-        const int i = t / p.kw, j = t - i * p.kw;
-        s_shift[t] = cfg.patch && t < cfg.taps ? (i * p.dil_h - p.pad_h) * p.w + (j * p.dil_w - p.pad_w) - cfg.lo : 0;
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -286,36 +295,44 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         // =========================== MMA issuers ===========================
         const int iss = warp < 4 ? warp - 2 : warp - 14;
         if (lane == 0 && iss < cfg.n_iss) {
-            const uint32_t idesc = umma_idesc_tf32(BM, T);
+            const uint32_t idesc = umma_idesc_tf32(BM, cfg.mma_n);
+            const int units_per_tile = T / cfg.mma_n;
             RingPos rw;
             uint32_t set = 0, set_par = 0;
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
+            // state of the next chunk's barriers, looked up while this chunk's MMAs are being issued
+            bool pre_w = false, pre_a = false;
             for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
-                if (acc_wrapped && !mbar_wait_lone(smem_u32(&s_accfree[ab]), acc_par ^ 1u)) {
+                if (acc_wrapped && !wait_or_abort(smem_u32(&s_accfree[ab]), acc_par ^ 1u, abort_flag)) {
                     *abort_flag = 5;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
                 for (int c = 0; c < n_chunks_item; ++c) {
-                    if (!mbar_wait_lone(smem_u32(&s_wfull[rw.s]), rw.parity)) { *abort_flag = 6; break; }
-                    if (!mbar_wait_lone(smem_u32(&s_aready[set]), set_par)) { *abort_flag = 7; break; }
-                    if (aborted(abort_flag)) break;
+                    if (!pre_w && !wait_or_abort(smem_u32(&s_wfull[rw.s]), rw.parity, abort_flag)) { *abort_flag = 6; break; }
+                    if (!pre_a && !wait_or_abort(smem_u32(&s_aready[set]), set_par, abort_flag)) { *abort_flag = 7; break; }
                     tc_fence_after();
                     const uint32_t b_smem = w_ring + rw.s * cfg.wstage_bytes;
                     const uint32_t a_set = tmem + A_COL0 + set * cfg.set_cols;
-                    for (int t = iss; t < g; t += cfg.n_iss) {
-                        const uint64_t bdesc = umma_desc_k_sw128(b_smem + t * T * 128, 1024);
-#pragma unroll
-                        for (int kq = 0; kq < P::KC / 8; ++kq)
-                            umma_tf32_ts(acc + t * T, a_set + t * cfg.kcp + kq * 8, bdesc + 2 * kq, idesc,
-                                         (c > 0 || kq > 0) ? 1u : 0u);
-                    }
-                    umma_commit(smem_u32(&s_afree[set]));
-                    umma_commit(smem_u32(&s_wfree[rw.s]));
+                    const uint32_t cur_w = smem_u32(&s_wfree[rw.s]), cur_a = smem_u32(&s_afree[set]);
                     rw.advance(cfg.n_w);
                     if (++set == static_cast<uint32_t>(cfg.n_sets)) { set = 0; set_par ^= 1u; }
+                    for (int u = iss; u < cfg.n_units; u += cfg.n_iss) {
+                        const uint64_t bdesc = umma_desc_k_sw128(b_smem + u * cfg.mma_n * 128, 1024);
+                        const uint32_t a_tile = a_set + (u / units_per_tile) * cfg.kcp;
+#pragma unroll
+                        for (int kq = 0; kq < P::KC / 8; ++kq)
+                            NM_CHECKED(((acc - tmem) & 0xFFFFu) + (u + 1) * cfg.mma_n <= 256u && ((a_tile - tmem) & 0xFFFFu) + kq * 8 + 8 <= 512u &&
+                                           b_smem + (u + 1) * cfg.mma_n * 128 <= staging && b_smem >= w_ring,
+                                       p.status, 801, u * 1000 + kq)
+                            umma_tf32_ts(acc + u * cfg.mma_n, a_tile + kq * 8, bdesc + 2 * kq, idesc, (c > 0 || kq > 0) ? 1u : 0u);
+                    }
+                    umma_commit(cur_a);
+                    umma_commit(cur_w);
+                    pre_w = mbar_test_wait(smem_u32(&s_wfull[rw.s]), rw.parity);
+                    pre_a = mbar_test_wait(smem_u32(&s_aready[set]), set_par);
                 }
                 if (aborted(abort_flag)) break;
                 umma_commit(smem_u32(&s_accfull[ab]));
@@ -401,20 +418,16 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         if (lane == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads; the writes complete with the grid
     } else if (warp >= 8 && warp < 16) {
         // =========================== compactors ===========================
-        const int wg = (warp - 8) >> 2;   // which half of the chunk
-        const int q = warp & 3;           // TMEM lane quadrant
+        const uint32_t team = static_cast<uint32_t>(warp - 8) >> 2;   // chunks cg = team (mod 2) are this warp's
+        const int q = warp & 3;                                       // TMEM lane quadrant
         const int row = q * 32 + lane;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t zero_row = smem_u32(s_zero);
-        // S = 64: half wg is 32-channel sub-tile wg; S = 32: half wg is the 16-byte pieces 4 wg .. 4 wg + 3 of the
-        // one sub-tile (a piece index enters the address XOR-ed with the row's swizzle phase)
-        const uint32_t half_off = P::SEGS == 2 ? static_cast<uint32_t>(wg) * cfg.seg_bytes : 0u;
-        const uint32_t half_piece = P::SEGS == 2 ? 0u : static_cast<uint32_t>(wg) * 4u;
-        const uint32_t im2col_row = static_cast<uint32_t>(row) * 128u + ((static_cast<uint32_t>(row & 7) ^ half_piece) << 4);
         const int hw = p.ho * p.wo;
         RingPos rp, rw;
         uint32_t set = 0, set_par = 0;
-        bool set_wrapped = false;
+        uint32_t cg = 0;                   // chunks of this CTA so far (all items)
+        bool pre_w = false, pre_a = false; // barriers of this team's next chunk found complete ahead of time
         for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
             const Item it = item_of(work, cfg);
             uint32_t vbits = 0xFFFFFFFFu;   // taps of this thread's pixel that lie inside the image
@@ -435,62 +448,104 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                     }
                 }
             }
-            for (int s = 0; s < cfg.n_act; ++s) {
-                bool ok = mbar_wait_lone(smem_u32(&s_pfull[rp.s]), rp.parity);
-                if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 3;
-                if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
-                const uint32_t act = p_ring + rp.s * cfg.p_bytes + half_off;
-                for (int t = 0; t < cfg.taps; ++t) {
-                    ok = mbar_wait_lone(smem_u32(&s_wfull[rw.s]), rw.parity);
-                    if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 10;
-                    ok = !set_wrapped || mbar_wait_lone(smem_u32(&s_afree[set]), set_par ^ 1u);
-                    if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 4;
-                    if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
+            bool failed = false;
+            for (int s = 0; s < cfg.n_act && !failed; ++s) {
+                const uint32_t act = p_ring + rp.s * cfg.p_bytes;
+                const uint32_t pfull = smem_u32(&s_pfull[rp.s]), pfree = smem_u32(&s_pfree[rp.s]);
+                const uint32_t ppar = rp.parity;
+                rp.advance(cfg.n_p);
+                bool stage_seen = false;
+                // patch form: rows between the first patch row and this pixel's source row of tap (ti, tj)
+                int shift_row = cfg.patch ? -p.pad_h * p.w - p.pad_w - cfg.lo : 0, shift = shift_row;
+                int tj = 0;
+                for (int t = 0; t < cfg.taps; ++t, ++cg) {
+                    const uint32_t my_shift = static_cast<uint32_t>(shift);
+                    shift += p.dil_w;
+                    if (++tj == p.kw) { tj = 0; shift_row += p.dil_h * p.w; shift = shift_row; }
+                    const uint32_t wst = w_ring + rw.s * cfg.wstage_bytes;
+                    const uint32_t wfull = smem_u32(&s_wfull[rw.s]), wfree = smem_u32(&s_wfree[rw.s]), wpar = rw.parity;
+                    const uint32_t aready = smem_u32(&s_aready[set]), afree = smem_u32(&s_afree[set]);
+                    const uint32_t a_set = tmem + lane_addr + A_COL0 + set * cfg.set_cols;
+                    const bool set_reused = cg >= static_cast<uint32_t>(cfg.n_sets);
+                    const uint32_t apar = set_par ^ 1u;
+                    rw.advance(cfg.n_w);
+                    if (++set == static_cast<uint32_t>(cfg.n_sets)) { set = 0; set_par ^= 1u; }
+                    if ((cg & 1u) != team) continue;
+                    bool ok = stage_seen || wait_or_abort(pfull, ppar, abort_flag);
+                    stage_seen = true;
+                    ok = ok && (pre_w || wait_or_abort(wfull, wpar, abort_flag));
+                    ok = ok && (!set_reused || pre_a || wait_or_abort(afree, apar, abort_flag));
+                    if (!__all_sync(0xFFFFFFFFu, ok)) { *abort_flag = 3; failed = true; break; }
                     tc_fence_after();
                     // address of this thread's row with the swizzle phase folded in: piece i lies at a0 ^ (i << 4)
-                    uint32_t a0;
-                    if (cfg.patch) {
-                        const uint32_t pr = static_cast<uint32_t>(row + s_shift[t]);
-                        a0 = ((vbits >> t) & 1u) ? act + pr * 128u + (((pr & 7u) ^ half_piece) << 4) : zero_row;
-                    } else {
-                        a0 = act + im2col_row;
+                    uint32_t a0 = zero_row;
+                    if (!cfg.patch) {
+                        a0 = act + static_cast<uint32_t>(row) * 128u + (static_cast<uint32_t>(row & 7) << 4);
+                    } else if ((vbits >> t) & 1u) {
+                        const uint32_t pr = static_cast<uint32_t>(row) + my_shift;
+                        a0 = act + pr * 128u + ((pr & 7u) << 4);
                     }
-                    uint32_t x[P::LW * 4];   // this half's S / 2 source columns of the row
+                    const bool live_row = a0 != zero_row;
 #pragma unroll
-                    for (int i = 0; i < P::LW; ++i) lds128(a0 ^ (static_cast<uint32_t>(i) << 4), x + 4 * i);
-                    const uint32_t mbase = w_ring + rw.s * cfg.wstage_bytes + cfg.w_bytes + wg * (P::HW * 4);
-                    const uint32_t a_set = tmem + lane_addr + A_COL0 + set * cfg.set_cols + wg * P::KW;
-                    for (int tile = 0; tile < g; ++tile) {
-                        uint32_t M[P::HW > 0 ? P::HW : 1];
+                    for (int half = 0; half < 2; ++half) {
+                        // S = 64: half h is 32-channel sub-tile h; S = 32: half h is the 16-byte pieces 4 h .. 4 h + 3 of the
+                        // one sub-tile (a piece index enters the address XOR-ed with the row's swizzle phase)
+                        const uint32_t ah = !live_row ? zero_row
+                                            : P::SEGS == 2 ? a0 + static_cast<uint32_t>(half) * cfg.seg_bytes
+                                                           : a0 ^ (static_cast<uint32_t>(half) << 6);
+                        uint32_t x[P::LW * 4];   // this half's S / 2 source columns of the row
 #pragma unroll
-                        for (int i = 0; i < P::HW / 4; ++i) lds128(mbase + tile * (P::MW * 4) + i * 16, M + 4 * i);
-                        uint32_t v[P::KW];
-#pragma unroll
-                        for (int gi = 0; gi < P::GW; ++gi) {
-#pragma unroll
-                            for (int j = 0; j < NK; ++j) {
-                                uint32_t r = x[gi * MG + j + P::D];
-#pragma unroll
-                                for (int i = P::D - 1; i >= 0; --i) r = bsel(M[(gi * NK + j) * P::D + i], x[gi * MG + j + i], r);
-                                v[gi * NK + j] = r;
-                            }
+                        for (int i = 0; i < P::LW; ++i) {
+                            x[4 * i] = x[4 * i + 1] = x[4 * i + 2] = x[4 * i + 3] = 0u;
+                            NM_CHECKED((ah >= p_ring && ah + 128u <= w_ring + 128u && (ah & 15u) == 0u) || (ah & ~127u) == zero_row, p.status, 802, ah)
+                            lds128(ah ^ (static_cast<uint32_t>(i) << 4), x + 4 * i);
                         }
-                        tmem_st_n<P::KW>(a_set + tile * cfg.kcp, v);
+                        if (half == 1) {
+                            // the barriers of this team's next chunk, looked up while the loads are in flight
+                            RingPos nw = rw;
+                            nw.advance(cfg.n_w);
+                            uint32_t nset = set + 1, npar = set_par;
+                            if (nset == static_cast<uint32_t>(cfg.n_sets)) { nset = 0; npar ^= 1u; }
+                            pre_w = mbar_test_wait(smem_u32(&s_wfull[nw.s]), nw.parity);
+                            pre_a = mbar_test_wait(smem_u32(&s_afree[nset]), npar ^ 1u);
+                        }
+                        const uint32_t mbase = wst + cfg.w_bytes + half * (P::HW * 4);
+                        for (int tile = 0; tile < g; ++tile) {
+                            uint32_t M[P::HW > 0 ? P::HW : 1];
+#pragma unroll
+                            for (int i = 0; i < P::HW / 4; ++i) {
+                                M[4 * i] = M[4 * i + 1] = M[4 * i + 2] = M[4 * i + 3] = 0u;
+                                NM_CHECKED(mbase + tile * (P::MW * 4) + i * 16 + 16 <= staging && mbase >= w_ring && (mbase & 15u) == 0u, p.status, 803, mbase)
+                                lds128(mbase + tile * (P::MW * 4) + i * 16, M + 4 * i);
+                            }
+                            uint32_t v[P::KW];
+#pragma unroll
+                            for (int gi = 0; gi < P::GW; ++gi) {
+#pragma unroll
+                                for (int j = 0; j < NK; ++j) {
+                                    uint32_t r = x[gi * MG + j + P::D];
+#pragma unroll
+                                    for (int i = P::D - 1; i >= 0; --i) r = bsel(M[(gi * NK + j) * P::D + i], x[gi * MG + j + i], r);
+                                    v[gi * NK + j] = r;
+                                }
+                            }
+                            NM_CHECKED(((a_set - tmem) & 0xFFFFu) + tile * cfg.kcp + half * P::KW + P::KW <= 512u &&
+                                           ((a_set - tmem) & 0xFFFFu) >= static_cast<uint32_t>(A_COL0) && ((a_set - tmem) >> 16) == static_cast<uint32_t>(q * 32),
+                                       p.status, 804, a_set - tmem)
+                            tmem_st_n<P::KW>(a_set + tile * cfg.kcp + half * P::KW, v);
+                        }
                     }
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) {
-                        mbar_arrive(smem_u32(&s_aready[set]));
-                        mbar_arrive(smem_u32(&s_wfree[rw.s]));
-                        if (t == cfg.taps - 1) mbar_arrive(smem_u32(&s_pfree[rp.s]));
+                        mbar_arrive(aready);
+                        mbar_arrive(wfree);
+                        if (t + 2 >= cfg.taps) mbar_arrive(pfree);   // this team's last chunk of the stage
                     }
-                    rw.advance(cfg.n_w);
-                    if (++set == static_cast<uint32_t>(cfg.n_sets)) { set = 0; set_par ^= 1u; set_wrapped = true; }
                 }
-                if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
-                rp.advance(cfg.n_p);
             }
+            if (failed) break;
         }
     }
 
@@ -592,12 +647,17 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     cfg->bn = g * T;
     cfg->n_slices = p.n_tiles / g;
     cfg->n_acc = cfg->bn <= 128 ? 2 : 1;
-    int n_iss = plan && plan->issuers > 0 ? plan->issuers : g;
-    if (n_iss > g || n_iss > MAX_ISS) return false;
+    // MMA units: the item's accumulator columns cut into up to four pieces, none across two tiles
+    int sub = g == 1 ? 4 : g == 2 ? 2 : 1;
+    while (sub > 1 && (T % sub != 0 || (T / sub) % 16 != 0)) sub /= 2;
+    cfg->mma_n = T / sub;
+    cfg->n_units = g * sub;
+    int n_iss = plan && plan->issuers > 0 ? plan->issuers : (cfg->n_units < MAX_ISS ? cfg->n_units : MAX_ISS);
+    if (n_iss > cfg->n_units || n_iss > MAX_ISS) return false;
     cfg->n_iss = n_iss;
     cfg->kcp = KC <= 8 ? 8 : KC <= 16 ? 16 : 32;
     cfg->set_cols = g * cfg->kcp;
-    cfg->n_sets = 256 / cfg->set_cols > MAX_SETS ? MAX_SETS : 256 / cfg->set_cols;
+    cfg->n_sets = 256 / cfg->set_cols >= MAX_SETS ? MAX_SETS : 2;   // 2 or 4: the two compactor teams alternate sets
     cfg->w_bytes = cfg->bn * 128;
     cfg->m_bytes = g * MW * 4;
     cfg->wstage_bytes = ((cfg->w_bytes + cfg->m_bytes + 1023) / 1024) * 1024;
@@ -612,14 +672,23 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
                        p.splitk_bytes < static_cast<size_t>(ksplit) * cfg->p_pad * p.c_out * sizeof(float) ||
                        static_cast<long long>(ksplit) * cfg->p_pad >= (1ll << 31)))
         return false;   // the partial-sum scratch is reserved by nm_autotune / nm_weights_reserve
-    // shared memory: two activation stages at least, the rest to the weight ring
+    // Shared memory: the activation ring, the rest to the weight ring.  The two compactor teams take alternate
+    // chunks and wait on a barrier by phase parity, so a team must meet EVERY use of a ring slot it waits on, or a
+    // wait for use k + 2 would pass on the completion of use k: the weight ring has an even number of slots (a slot
+    // always holds chunks of one parity, i.e. of one team), and so has the activation ring when a stage is one chunk
+    // (with several chunks per stage both teams read every stage).
     const int budget = 227 * 1024 - 1024 - STAGING_BYTES - 2048;   // alignment slack, output staging, static shared
-    int n_p = cfg->patch ? 2 : 3;
+    const bool paired = cfg->taps == 1;
+    int n_p = 2;
     if (plan && plan->stages > 0) n_p = plan->stages;
-    if (n_p < 1 || n_p > MAX_P) return false;
-    while (n_p > 1 && !(plan && plan->stages > 0) && n_p * cfg->p_bytes + 2 * cfg->wstage_bytes > budget) --n_p;
+    if (n_p < 1 || n_p > MAX_P || (paired && n_p % 2 != 0)) return false;
+    if (!(plan && plan->stages > 0)) {
+        if (paired && 4 * cfg->p_bytes + 4 * cfg->wstage_bytes <= budget) n_p = 4;
+        while (n_p > (paired ? 2 : 1) && n_p * cfg->p_bytes + 2 * cfg->wstage_bytes > budget) n_p -= paired ? 2 : 1;
+    }
     int n_w = (budget - n_p * cfg->p_bytes) / cfg->wstage_bytes;
     if (n_w > MAX_W) n_w = MAX_W;
+    n_w &= ~1;
     if (n_w < 2) return false;
     cfg->n_p = n_p;
     cfg->n_w = n_w;

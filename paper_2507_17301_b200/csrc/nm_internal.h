@@ -85,6 +85,26 @@ __device__ __forceinline__ void nm_add4(float4& a, const float4& b)
 }
 #endif
 
+#ifdef __CUDACC__
+// Self-checking build (-DNM_DEBUG_BOUNDS): the kernels that compute addresses from index data range-check
+// every such address; a violation is recorded in the handle's status word (error code NM_ERR_INTERNAL, the
+// site, the block, the offending value) and the access is skipped.  Nothing traps; nm_weights_check reports it.
+#ifdef NM_DEBUG_BOUNDS
+__device__ __forceinline__ void nm_debug_violation(int* status, int site, uint32_t value)
+{
+    if (atomicCAS(status + 0, 0, static_cast<int>(NM_ERR_INTERNAL)) == 0) {
+        atomicExch(status + 1, site);
+        atomicExch(status + 2, static_cast<int>(blockIdx.x));
+        atomicExch(status + 3, static_cast<int>(value));
+    }
+}
+#define NM_CHECKED(cond, status, site, value) \
+    if (!(cond)) nm_debug_violation((status), (site), static_cast<uint32_t>(value)); else
+#else
+#define NM_CHECKED(cond, status, site, value)
+#endif
+#endif
+
 namespace nmhost {
 // Launches `kernel` so that it may begin while the previous kernel of the stream drains
 // (programmatic dependent launch); the kernel orders itself with griddepcontrol.wait.

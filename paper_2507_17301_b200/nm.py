@@ -13,7 +13,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libnm_b200.so")
+# NM_LIBRARY selects another build of the same library (e.g. the self-checking libnm_b200_debug.so that
+# `python -m paper_2507_17301_b200.build -DNM_DEBUG_BOUNDS` makes)
+LIB_PATH = os.environ.get("NM_LIBRARY") or os.path.join(_HERE, "libnm_b200.so")
 
 NM_OK = 0
 NM_ERR_INVALID_ARG = -1

@@ -28,8 +28,8 @@ def _plan(nm, **kw):
 
 def _plans(nm, s):
     t = s.tile_t
-    return [_plan(nm), _plan(nm, loads=1), _plan(nm, loads=2), _plan(nm, bn=t), _plan(nm, bn=t, loads=1, stages=1),
-            _plan(nm, bn=2 * t, issuers=1), _plan(nm, bn=4 * t, issuers=2, loads=1), _plan(nm, bn=4 * t, loads=2, stages=1),
+    return [_plan(nm), _plan(nm, loads=1), _plan(nm, loads=2), _plan(nm, bn=t), _plan(nm, bn=t, loads=1, stages=2),
+            _plan(nm, bn=2 * t, issuers=1), _plan(nm, bn=4 * t, issuers=2, loads=1), _plan(nm, bn=4 * t, loads=2, stages=1), _plan(nm, loads=1, stages=4),
             _plan(nm, bn=256), _plan(nm, bn=128, loads=2)]
 
 
