@@ -48,7 +48,6 @@ namespace {
 using namespace nmk;
 
 constexpr int BM = 128;
-constexpr int SUB_BYTES = BM * 128;
 constexpr int THREADS = 576;   // warps: 0 activation producer, 1 weight producer, 2 3 16 17 MMA issuers, 4-7 epilogue, 8-15 compactors
 constexpr int MAX_P = 4;       // activation ring slots
 constexpr int MAX_W = 8;       // weight ring slots
@@ -73,6 +72,8 @@ struct SelCfg {
     int wstage_bytes;   // w_bytes + m_bytes rounded up to 1024
     int n_p, n_w, n_sets, kcp, set_cols;
     int ksplit, p_pad;
+    int alias_staging;  // 1: the output staging boxes lie over the start of the activation ring (one work item per CTA)
+    int boxes;          // staging boxes (32 pixels x 32 channels) per epilogue warp: 2, or one per channel block when aliased
     int n_act;          // activation stages per work item
     long long n_work;
 };
@@ -95,6 +96,31 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 __device__ __forceinline__ void lds128(uint32_t addr, uint32_t* dst)
 {
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(dst[0]), "=r"(dst[1]), "=r"(dst[2]), "=r"(dst[3]) : "r"(addr));
+}
+// `n` consecutive 32-bit words of shared memory (n a compile-time constant, addr aligned to `align` bytes).
+template <int N, int ALIGN>
+__device__ __forceinline__ void lds_words(uint32_t addr, uint32_t* dst)
+{
+    if constexpr (ALIGN % 16 == 0 && N % 4 == 0) {
+#pragma unroll
+        for (int i = 0; i < N / 4; ++i) lds128(addr + 16 * i, dst + 4 * i);
+    } else if constexpr (ALIGN % 8 == 0 && N % 2 == 0) {
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i)
+            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(dst[2 * i]), "=r"(dst[2 * i + 1]) : "r"(addr + 8 * i));
+    } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(dst[i]) : "r"(addr + 4 * i));
+    }
+}
+// Byte `k` of `w` (0x80 = set, 0x00 = clear) widened to a 32-bit mask of all ones / all zeros: one byte permute
+// whose four selectors replicate the sign bit of the chosen byte.
+template <int K>
+__device__ __forceinline__ uint32_t mask_of_byte(uint32_t w)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(d) : "r"(w), "n"(0x8888 | (0x1111 * K)));
+    return d;
 }
 // m ? a : b, bit by bit (m is all ones or all zeros)
 __device__ __forceinline__ uint32_t bsel(uint32_t m, uint32_t a, uint32_t b)
@@ -131,8 +157,9 @@ struct Pattern {
     static constexpr int GW = GROUPS / 2;                    // groups per compactor half
     static constexpr int KW = GW * NK;                       // kept columns per compactor half
     static constexpr int LW = S / 8;                         // 16-byte pieces of a row per compactor half
-    static constexpr int MW = GROUPS * NK * D;               // mask words per tile and chunk
-    static constexpr int HW = MW / 2;                        // ... per compactor half
+    static constexpr int MW = GROUPS * NK * D;               // select masks (one byte each) per tile and chunk
+    static constexpr int HW = MW / 2;                        // ... per half of the chunk
+    static constexpr int MWP = (MW + 15) / 16 * 16;          // bytes a tile's masks of one chunk occupy (bulk copies move 16-byte units)
 };
 
 struct Item {
@@ -156,9 +183,10 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
 {
     using P = Pattern<NK, MG>;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t s_pfull[MAX_P], s_pfree[MAX_P], s_wfull[MAX_W], s_wfree[MAX_W], s_aready[MAX_SETS],
-        s_afree[MAX_SETS], s_accfull[2], s_accfree[2];
-    __shared__ __align__(128) float s_zero[32];
+    __shared__ uint64_t s_pfull[MAX_P], s_pfree[MAX_P], s_wfull[MAX_W], s_wfree[MAX_W], s_aready[MAX_SETS], s_accfull[2],
+        s_accfree[2];
+    __shared__ __align__(1024) float s_zero[8 * 32];   // eight rows of zeros, one per swizzle phase (an out-of-image tap reads
+                                                          // the row of its own phase: no bank conflict with its neighbours)
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
 
@@ -167,7 +195,9 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
     const int T = p.tile_t, g = cfg.g;
     const uint32_t p_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t w_ring = p_ring + cfg.n_p * cfg.p_bytes;
-    const uint32_t staging = w_ring + cfg.n_w * cfg.wstage_bytes;
+    const uint32_t ring_end = w_ring + cfg.n_w * cfg.wstage_bytes;
+    // with one work item per CTA the epilogue starts when every load has been consumed: its staging boxes reuse the ring
+    const uint32_t staging = cfg.alias_staging ? p_ring : ring_end;
     const int n_chunks_item = cfg.n_act * cfg.taps;
     volatile int* abort_flag = &s_abort;
 
@@ -180,11 +210,13 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         }
         for (int i = 0; i < MAX_W; ++i) {
             mbar_init(smem_u32(&s_wfull[i]), 1);
-            mbar_init(smem_u32(&s_wfree[i]), 4 + cfg.n_iss);  // one compactor team (masks) + MMA commits (weights)
+            // one compactor team (it has read the masks) + one MMA commit per issuer (the weights and the operand set
+            // have been read): the weight producer waits on it before refilling the slot, a compactor team before it
+            // overwrites the operand set that chunk used
+            mbar_init(smem_u32(&s_wfree[i]), 4 + cfg.n_iss);
         }
         for (int i = 0; i < MAX_SETS; ++i) {
-            mbar_init(smem_u32(&s_aready[i]), 4);             // one compactor team
-            mbar_init(smem_u32(&s_afree[i]), cfg.n_iss);      // MMA commits
+            mbar_init(smem_u32(&s_aready[i]), 4);             // one compactor team: operand set written AND weights landed
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&s_accfull[i]), cfg.n_iss);
@@ -195,7 +227,7 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         tma_prefetch_desc(&tm_x);
         tma_prefetch_desc(&tm_y);
     }
-    if (tid < 32) s_zero[tid] = 0.f;
+    if (tid < 8 * 32) s_zero[tid] = 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -220,6 +252,12 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                 int tap = 0, cb = a;                       // im2col: stage a = chunk a = (tap, cb)
                 if (!cfg.patch) { tap = a / cfg.n_cb; cb = a - tap * cfg.n_cb; }
                 int ti = tap / p.kw, tj = tap - ti * p.kw;
+                if (cfg.patch) {
+                    // the item's activations, all channel blocks: out of HBM now, not one ring slot at a time
+                    for (int s = cfg.n_p; s < cfg.n_act; ++s)
+                        for (int seg = 0; seg < P::SEGS; ++seg)
+                            l2_prefetch_tile_2d(&tm_x, ((a + s) * P::SEGS + seg) * 32, static_cast<int>(it.pix0) + cfg.lo);
+                }
                 for (int s = 0; s < cfg.n_act; ++s) {
                     if (rp.wrapped && !mbar_wait_lone(smem_u32(&s_pfree[rp.s]), rp.parity ^ 1u)) *abort_flag = 2;
                     if (aborted(abort_flag)) break;
@@ -258,12 +296,12 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
             RingPos rw;
             int issued = 0;
             const size_t chunk_floats = static_cast<size_t>(p.c_out) * 32;
-            const size_t chunk_words = static_cast<size_t>(p.n_tiles) * P::MW;
+            const size_t chunk_mbytes = static_cast<size_t>(p.n_tiles) * P::MWP;
             const uint32_t tx = static_cast<uint32_t>(cfg.w_bytes + cfg.m_bytes);
             for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 const Item it = item_of(work, cfg);
                 const float* wsl = p.w3 + static_cast<size_t>(it.slice) * cfg.bn * 32;
-                const uint32_t* msl = p.sel3 + static_cast<size_t>(it.slice) * g * P::MW;
+                const uint8_t* msl = p.sel3 + static_cast<size_t>(it.slice) * g * P::MWP;
                 const int a0 = it.split * cfg.n_act;
                 for (int s = 0; s < cfg.n_act && !aborted(abort_flag); ++s) {
                     // patch: stage = channel block a0 + s, its chunks are (tap, block) for every tap; im2col: chunk a0 + s
@@ -276,7 +314,7 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                         mbar_arrive_expect_tx(bar, tx);
                         bulk_load_1d(dst, wsl + static_cast<size_t>(c) * chunk_floats, static_cast<uint32_t>(cfg.w_bytes), bar);
                         if (P::MW > 0)
-                            bulk_load_1d(dst + cfg.w_bytes, msl + static_cast<size_t>(c) * chunk_words,
+                            bulk_load_1d(dst + cfg.w_bytes, msl + static_cast<size_t>(c) * chunk_mbytes,
                                          static_cast<uint32_t>(cfg.m_bytes), bar);
                         rw.advance(cfg.n_w);
                         ++issued;
@@ -301,8 +339,9 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
             uint32_t set = 0, set_par = 0;
             uint32_t ab = 0, acc_par = 0;
             bool acc_wrapped = false;
-            // state of the next chunk's barriers, looked up while this chunk's MMAs are being issued
-            bool pre_w = false, pre_a = false;
+            // A chunk is ready when its compactor team has arrived: the team waits for the chunk's weights (they
+            // come with its masks) before it starts, so this one barrier stands for both.  One commit per chunk
+            // releases the weight slot and, through the same barrier, the operand set.
             for (uint32_t work = blockIdx.x; work < n_work && !aborted(abort_flag); work += gridDim.x) {
                 if (acc_wrapped && !wait_or_abort(smem_u32(&s_accfree[ab]), acc_par ^ 1u, abort_flag)) {
                     *abort_flag = 5;
@@ -311,28 +350,23 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                 tc_fence_after();
                 const uint32_t acc = tmem + ab * cfg.bn;
                 for (int c = 0; c < n_chunks_item; ++c) {
-                    if (!pre_w && !wait_or_abort(smem_u32(&s_wfull[rw.s]), rw.parity, abort_flag)) { *abort_flag = 6; break; }
-                    if (!pre_a && !wait_or_abort(smem_u32(&s_aready[set]), set_par, abort_flag)) { *abort_flag = 7; break; }
+                    if (!wait_or_abort(smem_u32(&s_aready[set]), set_par, abort_flag)) { *abort_flag = 7; break; }
                     tc_fence_after();
                     const uint32_t b_smem = w_ring + rw.s * cfg.wstage_bytes;
                     const uint32_t a_set = tmem + A_COL0 + set * cfg.set_cols;
-                    const uint32_t cur_w = smem_u32(&s_wfree[rw.s]), cur_a = smem_u32(&s_afree[set]);
-                    rw.advance(cfg.n_w);
-                    if (++set == static_cast<uint32_t>(cfg.n_sets)) { set = 0; set_par ^= 1u; }
                     for (int u = iss; u < cfg.n_units; u += cfg.n_iss) {
                         const uint64_t bdesc = umma_desc_k_sw128(b_smem + u * cfg.mma_n * 128, 1024);
                         const uint32_t a_tile = a_set + (u / units_per_tile) * cfg.kcp;
 #pragma unroll
                         for (int kq = 0; kq < P::KC / 8; ++kq)
                             NM_CHECKED(((acc - tmem) & 0xFFFFu) + (u + 1) * cfg.mma_n <= 256u && ((a_tile - tmem) & 0xFFFFu) + kq * 8 + 8 <= 512u &&
-                                           b_smem + (u + 1) * cfg.mma_n * 128 <= staging && b_smem >= w_ring,
+                                           b_smem + (u + 1) * cfg.mma_n * 128 <= ring_end && b_smem >= w_ring,
                                        p.status, 801, u * 1000 + kq)
                             umma_tf32_ts(acc + u * cfg.mma_n, a_tile + kq * 8, bdesc + 2 * kq, idesc, (c > 0 || kq > 0) ? 1u : 0u);
                     }
-                    umma_commit(cur_a);
-                    umma_commit(cur_w);
-                    pre_w = mbar_test_wait(smem_u32(&s_wfull[rw.s]), rw.parity);
-                    pre_a = mbar_test_wait(smem_u32(&s_aready[set]), set_par);
+                    umma_commit(smem_u32(&s_wfree[rw.s]));
+                    rw.advance(cfg.n_w);
+                    if (++set == static_cast<uint32_t>(cfg.n_sets)) { set = 0; set_par ^= 1u; }
                 }
                 if (aborted(abort_flag)) break;
                 umma_commit(smem_u32(&s_accfull[ab]));
@@ -349,7 +383,7 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         // =========================== epilogue ===========================
         const int q = warp & 3;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const uint32_t my_staging = staging + q * 2 * 4096;
+        const uint32_t my_staging = staging + q * cfg.boxes * 4096;
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t ti = 0;
@@ -379,8 +413,9 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
                 }
-                const uint32_t box = my_staging + (nb & 1u) * 4096;
-                if (lane == 0 && nb >= 2) tma_store_wait_read_n<1>();  // the box's previous store has read it
+                // two boxes: the box's previous store (two blocks ago) has read it; a box per block: nothing to wait for
+                const uint32_t box = my_staging + (cfg.boxes == 2 ? (nb & 1u) : static_cast<uint32_t>(blk)) * 4096;
+                if (cfg.boxes == 2 && lane == 0 && nb >= 2) tma_store_wait_read_n<1>();
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
                 const bool res_pass = p.residual != nullptr && box_pix < p.pixels;
@@ -424,7 +459,7 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t zero_row = smem_u32(s_zero);
         const int hw = p.ho * p.wo;
-        RingPos rp, rw;
+        RingPos rp, rw, rold;              // rold: weight slot of the chunk n_sets chunks back
         uint32_t set = 0, set_par = 0;
         uint32_t cg = 0;                   // chunks of this CTA so far (all items)
         bool pre_w = false, pre_a = false; // barriers of this team's next chunk found complete ahead of time
@@ -464,10 +499,12 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                     if (++tj == p.kw) { tj = 0; shift_row += p.dil_h * p.w; shift = shift_row; }
                     const uint32_t wst = w_ring + rw.s * cfg.wstage_bytes;
                     const uint32_t wfull = smem_u32(&s_wfull[rw.s]), wfree = smem_u32(&s_wfree[rw.s]), wpar = rw.parity;
-                    const uint32_t aready = smem_u32(&s_aready[set]), afree = smem_u32(&s_afree[set]);
+                    const uint32_t aready = smem_u32(&s_aready[set]);
                     const uint32_t a_set = tmem + lane_addr + A_COL0 + set * cfg.set_cols;
+                    // the operand set was last used by chunk cg - n_sets: its MMAs are done when its weight slot is free
                     const bool set_reused = cg >= static_cast<uint32_t>(cfg.n_sets);
-                    const uint32_t apar = set_par ^ 1u;
+                    const uint32_t afree = smem_u32(&s_wfree[rold.s]), apar = rold.parity;
+                    if (set_reused) rold.advance(cfg.n_w);
                     rw.advance(cfg.n_w);
                     if (++set == static_cast<uint32_t>(cfg.n_sets)) { set = 0; set_par ^= 1u; }
                     if ((cg & 1u) != team) continue;
@@ -478,46 +515,40 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                     if (!__all_sync(0xFFFFFFFFu, ok)) { *abort_flag = 3; failed = true; break; }
                     tc_fence_after();
                     // address of this thread's row with the swizzle phase folded in: piece i lies at a0 ^ (i << 4)
-                    uint32_t a0 = zero_row;
-                    if (!cfg.patch) {
-                        a0 = act + static_cast<uint32_t>(row) * 128u + (static_cast<uint32_t>(row & 7) << 4);
-                    } else if ((vbits >> t) & 1u) {
-                        const uint32_t pr = static_cast<uint32_t>(row) + my_shift;
-                        a0 = act + pr * 128u + ((pr & 7u) << 4);
-                    }
-                    const bool live_row = a0 != zero_row;
+                    const uint32_t pr = static_cast<uint32_t>(row) + (cfg.patch ? my_shift : 0u);
+                    const bool live_row = !cfg.patch || ((vbits >> t) & 1u);
+                    const uint32_t a0 = (live_row ? act + pr * 128u : zero_row + (pr & 7u) * 128u) + ((pr & 7u) << 4);
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         // S = 64: half h is 32-channel sub-tile h; S = 32: half h is the 16-byte pieces 4 h .. 4 h + 3 of the
                         // one sub-tile (a piece index enters the address XOR-ed with the row's swizzle phase)
-                        const uint32_t ah = !live_row ? zero_row
-                                            : P::SEGS == 2 ? a0 + static_cast<uint32_t>(half) * cfg.seg_bytes
-                                                           : a0 ^ (static_cast<uint32_t>(half) << 6);
+                        const uint32_t ah = P::SEGS == 1 ? a0 ^ (static_cast<uint32_t>(half) << 6)
+                                            : live_row   ? a0 + static_cast<uint32_t>(half) * cfg.seg_bytes
+                                                         : a0;
                         uint32_t x[P::LW * 4];   // this half's S / 2 source columns of the row
 #pragma unroll
                         for (int i = 0; i < P::LW; ++i) {
                             x[4 * i] = x[4 * i + 1] = x[4 * i + 2] = x[4 * i + 3] = 0u;
-                            NM_CHECKED((ah >= p_ring && ah + 128u <= w_ring + 128u && (ah & 15u) == 0u) || (ah & ~127u) == zero_row, p.status, 802, ah)
+                            NM_CHECKED((ah >= p_ring && ah + 128u <= w_ring + 128u && (ah & 15u) == 0u) || (ah & ~1023u) == zero_row, p.status, 802, ah)
                             lds128(ah ^ (static_cast<uint32_t>(i) << 4), x + 4 * i);
                         }
                         if (half == 1) {
                             // the barriers of this team's next chunk, looked up while the loads are in flight
-                            RingPos nw = rw;
+                            RingPos nw = rw, no = rold;
                             nw.advance(cfg.n_w);
-                            uint32_t nset = set + 1, npar = set_par;
-                            if (nset == static_cast<uint32_t>(cfg.n_sets)) { nset = 0; npar ^= 1u; }
+                            if (cg + 1 >= static_cast<uint32_t>(cfg.n_sets)) no.advance(cfg.n_w);
                             pre_w = mbar_test_wait(smem_u32(&s_wfull[nw.s]), nw.parity);
-                            pre_a = mbar_test_wait(smem_u32(&s_afree[nset]), npar ^ 1u);
+                            pre_a = mbar_test_wait(smem_u32(&s_wfree[no.s]), no.parity);
                         }
-                        const uint32_t mbase = wst + cfg.w_bytes + half * (P::HW * 4);
+                        const uint32_t mbase = wst + cfg.w_bytes + half * P::HW;
                         for (int tile = 0; tile < g; ++tile) {
-                            uint32_t M[P::HW > 0 ? P::HW : 1];
+                            constexpr int MWORDS = (P::HW + 3) / 4;
+                            constexpr int MALIGN = P::HW % 16 == 0 ? 16 : P::HW % 8 == 0 ? 8 : 4;
+                            uint32_t M[MWORDS];   // this half's select masks of the tile, one byte each
 #pragma unroll
-                            for (int i = 0; i < P::HW / 4; ++i) {
-                                M[4 * i] = M[4 * i + 1] = M[4 * i + 2] = M[4 * i + 3] = 0u;
-                                NM_CHECKED(mbase + tile * (P::MW * 4) + i * 16 + 16 <= staging && mbase >= w_ring && (mbase & 15u) == 0u, p.status, 803, mbase)
-                                lds128(mbase + tile * (P::MW * 4) + i * 16, M + 4 * i);
-                            }
+                            for (int i = 0; i < MWORDS; ++i) M[i] = 0u;
+                            NM_CHECKED(mbase + tile * P::MWP + MWORDS * 4 <= ring_end && mbase >= w_ring && (mbase & 3u) == 0u, p.status, 803, mbase)
+                            lds_words<MWORDS, MALIGN>(mbase + tile * P::MWP, M);
                             uint32_t v[P::KW];
 #pragma unroll
                             for (int gi = 0; gi < P::GW; ++gi) {
@@ -525,7 +556,17 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                                 for (int j = 0; j < NK; ++j) {
                                     uint32_t r = x[gi * MG + j + P::D];
 #pragma unroll
-                                    for (int i = P::D - 1; i >= 0; --i) r = bsel(M[(gi * NK + j) * P::D + i], x[gi * MG + j + i], r);
+                                    for (int i = P::D - 1; i >= 0; --i) {
+                                        const int mi = (gi * NK + j) * P::D + i;
+                                        uint32_t m;
+                                        switch (mi & 3) {
+                                            case 0: m = mask_of_byte<0>(M[mi >> 2]); break;
+                                            case 1: m = mask_of_byte<1>(M[mi >> 2]); break;
+                                            case 2: m = mask_of_byte<2>(M[mi >> 2]); break;
+                                            default: m = mask_of_byte<3>(M[mi >> 2]); break;
+                                        }
+                                        r = bsel(m, x[gi * MG + j + i], r);
+                                    }
                                     v[gi * NK + j] = r;
                                 }
                             }
@@ -589,7 +630,7 @@ void pattern_dims(int* s, int* kc, int* mw)
 {
     *s = Pattern<NK, MG>::S;
     *kc = Pattern<NK, MG>::KC;
-    *mw = Pattern<NK, MG>::MW;
+    *mw = Pattern<NK, MG>::MWP;
 }
 
 bool dims_of(int code, int* s, int* kc, int* mw)
@@ -659,7 +700,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     cfg->set_cols = g * cfg->kcp;
     cfg->n_sets = 256 / cfg->set_cols >= MAX_SETS ? MAX_SETS : 2;   // 2 or 4: the two compactor teams alternate sets
     cfg->w_bytes = cfg->bn * 128;
-    cfg->m_bytes = g * MW * 4;
+    cfg->m_bytes = g * MW;
     cfg->wstage_bytes = ((cfg->w_bytes + cfg->m_bytes + 1023) / 1024) * 1024;
     // split of the reduction axis: whole activation stages per range
     const int ksplit = plan && plan->ksplit > 1 ? plan->ksplit : 1;
@@ -677,7 +718,12 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     // wait for use k + 2 would pass on the completion of use k: the weight ring has an even number of slots (a slot
     // always holds chunks of one parity, i.e. of one team), and so has the activation ring when a stage is one chunk
     // (with several chunks per stage both teams read every stage).
-    const int budget = 227 * 1024 - 1024 - STAGING_BYTES - 2048;   // alignment slack, output staging, static shared
+    const long long pix_blocks = (p.pixels + BM - 1) / BM;
+    cfg->n_work = pix_blocks * cfg->n_slices * ksplit;
+    if (cfg->n_work >= (1ll << 31)) return false;
+    cfg->alias_staging = cfg->n_work <= sm_count();
+    // alignment slack, static shared, and the output staging unless it can lie over the ring
+    const int budget = 227 * 1024 - 1024 - 2048 - (cfg->alias_staging ? 0 : STAGING_BYTES);
     const bool paired = cfg->taps == 1;
     int n_p = 2;
     if (plan && plan->stages > 0) n_p = plan->stages;
@@ -692,9 +738,15 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     if (n_w < 2) return false;
     cfg->n_p = n_p;
     cfg->n_w = n_w;
-    const long long pix_blocks = (p.pixels + BM - 1) / BM;
-    cfg->n_work = pix_blocks * cfg->n_slices * ksplit;
-    if (cfg->n_work >= (1ll << 31)) return false;
+    // a set is released through the weight slot of the chunk that used it: the slot must not come round again sooner
+    if (cfg->n_sets > n_w) cfg->n_sets = n_w >= 4 ? 4 : 2;
+    cfg->boxes = 2;
+    if (cfg->alias_staging) {
+        // one work item per CTA: the rings are idle when the epilogue runs, every channel block gets a box of its own
+        const int ring_bytes = n_p * cfg->p_bytes + n_w * cfg->wstage_bytes;
+        if (ring_bytes >= 4 * (cfg->bn / 32) * 4096) cfg->boxes = cfg->bn / 32;
+        else if (ring_bytes < STAGING_BYTES) cfg->alias_staging = 0;
+    }
     return true;
 }
 
@@ -726,7 +778,8 @@ nm_status_t launch(const ConvParams& p, const SelCfg& cfg, cudaStream_t st)
     if (!ok_x || !nmtm::encode_y_tiled(q, &tm_y))
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 8)");
     q.pixels = p.pixels;
-    size_t smem = 1024 + static_cast<size_t>(cfg.n_p) * cfg.p_bytes + static_cast<size_t>(cfg.n_w) * cfg.wstage_bytes + STAGING_BYTES;
+    size_t smem = 1024 + static_cast<size_t>(cfg.n_p) * cfg.p_bytes + static_cast<size_t>(cfg.n_w) * cfg.wstage_bytes +
+                  (cfg.alias_staging ? 0 : STAGING_BYTES);
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
     cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_select<NK, MG>), smem);
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 8): %s", cudaGetErrorString(e));
@@ -756,10 +809,10 @@ __global__ void k_build_w3(const float* __restrict__ values, const uint16_t* __r
         nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
 }
 
-// Select masks: for retained column j (the jn-th of its group, at position pos in the group) the D = M - N words
-// m[i] = all ones iff pos == jn + i, i < D (all zero: the column is the last candidate, jn + D).
+// Select masks: for retained column j (the jn-th of its group, at position pos in the group) the D = M - N bytes
+// m[i] = 0x80 iff pos == jn + i, i < D (all zero: the column is the last candidate, jn + D); `mw` bytes per tile and chunk.
 __global__ void k_build_sel3(const uint16_t* __restrict__ indices, int n_tiles, int kk, int n_keep, int m_group,
-                             int s_cols, int kc, int mw, uint32_t* __restrict__ sel3)
+                             int s_cols, int kc, int mw, uint8_t* __restrict__ sel3)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     const int r = blockIdx.y;
@@ -770,8 +823,8 @@ __global__ void k_build_sel3(const uint16_t* __restrict__ indices, int n_tiles, 
     const int jj = j - chunk * kc;           // slot within the chunk = group-in-chunk * N + jn
     const int jn = jj % n_keep;
     const int pos = col % m_group;
-    uint32_t* m = sel3 + (static_cast<size_t>(chunk) * n_tiles + r) * mw + static_cast<size_t>(jj) * d;
-    for (int i = 0; i < d; ++i) m[i] = (pos == jn + i) ? 0xFFFFFFFFu : 0u;
+    uint8_t* m = sel3 + (static_cast<size_t>(chunk) * n_tiles + r) * mw + static_cast<size_t>(jj) * d;
+    for (int i = 0; i < d; ++i) m[i] = (pos == jn + i) ? 0x80u : 0u;
 }
 
 }  // namespace
@@ -792,7 +845,7 @@ nm_status_t build_select_layout(nm_weights* h, cudaStream_t st)
         return NM_OK;
     const int chunks = h->k / S;
     const size_t wbytes = static_cast<size_t>(chunks) * h->c_out * 32 * sizeof(float);
-    const size_t mbytes = static_cast<size_t>(chunks) * h->n_tiles * MW * sizeof(uint32_t);
+    const size_t mbytes = static_cast<size_t>(chunks) * h->n_tiles * MW;
     if (cudaMalloc(&h->w3, wbytes) != cudaSuccess || cudaMalloc(&h->sel3, mbytes) != cudaSuccess) {
         (void)cudaGetLastError();
         cudaFree(h->w3);
@@ -801,6 +854,7 @@ nm_status_t build_select_layout(nm_weights* h, cudaStream_t st)
         return fail(NM_ERR_ALLOC, "cannot allocate the select-kernel weights");
     }
     cudaError_t e = cudaMemsetAsync(h->w3, 0, wbytes, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->sel3, 0, mbytes, st);   // the padding bytes of a tile's masks
     if (e != cudaSuccess) return fail(NM_ERR_CUDA, "select layout memset: %s", cudaGetErrorString(e));
     const dim3 gw((h->kk + 127) / 128, h->c_out), gm((h->kk + 127) / 128, h->n_tiles);
     k_build_w3<<<gw, 128, 0, st>>>(h->values, h->indices, h->c_out, h->kk, h->tile_t, S, KC, h->w3);

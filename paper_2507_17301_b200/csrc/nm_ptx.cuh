@@ -237,6 +237,17 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// Prefetch into L2 (nothing lands in shared memory, nothing to wait for): a contiguous range (16-byte aligned,
+// a multiple of 16 bytes) or the box of a tiled tensor map.  Used to pull operands that every CTA of a launch
+// will stream in lockstep (weights above all) out of HBM ahead of the first load that needs them.
+__device__ __forceinline__ void l2_prefetch_1d(const void* src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void l2_prefetch_tile_2d(const void* tmap, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
+}
 // Shared -> global tiled store (bulk async group); rows / columns outside the tensor are clipped.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int x, int y)
 {
