@@ -39,10 +39,12 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 TF32_OVER_BF16 = 1.1 / 2.25   # nominal dense tensor peaks: 1.1 PFLOP/s TF32, 2.25 PFLOP/s bf16
 KERNEL_OF_VARIANT = {1: "k_conv_gather", 2: "k_conv_slab", 3: "k_conv_stream", 4: "k_conv_expand", 5: "k_conv_rowrun",
-                     6: "k_conv_window", 7: "k_conv_pair"}
+                     6: "k_conv_window", 7: "k_conv_pair", 8: "k_conv_select"}
 KERNEL_SOURCE = {"k_conv_gather": "nm_conv_gather.cu", "k_conv_slab": "nm_conv_slab.cu", "k_conv_stream": "nm_conv_stream.cu",
                  "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu", "k_conv_window": "nm_conv_window.cu",
-                 "k_conv_pair": "nm_conv_pair.cu"}
+                 "k_conv_pair": "nm_conv_pair.cu", "k_conv_select": "nm_conv_select.cu"}
+KEPT_ONLY_VARIANTS = (1, 2, 3, 8)   # kernels that contract over the retained columns only (Algorithm 1 proper)
+PLAN_FIELDS = ("variant", "bn", "stages", "split", "kblk", "loads", "issuers", "ksplit")
 
 
 def peaks():
@@ -275,29 +277,44 @@ def run_reference(args):
     }))
 
 
-def cpu_baseline(budget_s: float = 20.0):
+REL_FRO_TOL = 2e-3      # relative Frobenius error allowed under TF32
+MAX_ABS_TOL = 1e-2      # max-abs error allowed, as a fraction of max|ref|
+
+
+def parity_and_cpu_baseline(nm, state):
+    """Every layer under the plan that is about to be timed against the CPU checker on the bench's own
+    tensors: pruning bit for bit, image 0 of the output within the TF32 tolerance.  The checker's
+    convolutions are timed on the way: they are the `cpu_baseline` sample.  Runs outside the timed region."""
+    import numpy as np
     import oracle
-    layers = workload(1)
-    t_total, done = 0.0, 0
-    t_begin = time.perf_counter()
-    for li, s in enumerate(layers):
-        w = inputs.make_weights(s, li)
-        values, indices = oracle.prune(w.numpy(), s.n_keep, s.m_group, s.tile_t)
-        x = inputs.make_activations(s, li, batch=1).numpy()
-        b = inputs.make_bias(s, li).numpy()
+    worst_rel, worst_abs, t_total = 0.0, 0.0, 0.0
+    failed, prune_ok = [], True
+    for li, (s, hnd, x, bias, y, plan) in enumerate(state):
+        nm.nm_conv2d(hnd, x, s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=y, plan=plan)
+        nm.nm_weights_check(hnd)
+        v, i = nm.nm_weights_export(hnd)
+        torch.cuda.synchronize()
+        vr, ir = oracle.prune(inputs.make_weights(s, li).numpy(), s.n_keep, s.m_group, s.tile_t)
+        if not (np.array_equal(i.cpu().numpy(), ir) and np.array_equal(v.cpu().numpy().view(np.uint32), vr.view(np.uint32))):
+            prune_ok = False
+            failed.append(s.name + " (pruning)")
+        x0, b0 = x[0:1].cpu().numpy(), bias.cpu().numpy()
         t0 = time.perf_counter()
-        oracle.conv2d(values, indices, s.kh, s.kw, s.c_in, s.tile_t, x, (s.stride,) * 2, (s.pad,) * 2, (s.dil,) * 2, b,
-                      s.relu)
+        yr = oracle.conv2d(vr, ir, s.kh, s.kw, s.c_in, s.tile_t, x0, (s.stride,) * 2, (s.pad,) * 2, (s.dil,) * 2, b0, s.relu)
         t_total += time.perf_counter() - t0
-        done += 1
-        if time.perf_counter() - t_begin > budget_s * 3:
-            break
-    flops_done = sum(useful_flops(s) for s in layers[:done])
-    flops_all = sum(useful_flops(s) for s in layers)
-    est_image_s = t_total * flops_all / flops_done  # scaled by kept FLOPs if the budget cut the pass short
-    sample = (f"image 0 of the first {done} of {len(layers)} layers (1 image of the batch)"
-              + ("" if done == len(layers) else ", scaled to the stack by kept FLOPs"))
-    return {"value": 1.0 / est_image_s, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample}
+        d = y[0:1].cpu().numpy().astype(np.float64) - yr.astype(np.float64)
+        ref_n = float(np.sqrt((yr.astype(np.float64) ** 2).sum()))
+        rel = float(np.sqrt((d ** 2).sum())) / max(ref_n, 1e-30)
+        mx = float(np.abs(d).max()) / max(float(np.abs(yr).max()), 1e-30)
+        worst_rel, worst_abs = max(worst_rel, rel), max(worst_abs, mx)
+        if not (np.isfinite(d).all() and rel <= REL_FRO_TOL and mx <= MAX_ABS_TOL):
+            failed.append(s.name)
+    sample = f"image 0 of each of the {len(state)} layers (1 image of the batch), the bench's own tensors"
+    parity = {"layers": len(state), "max_rel_fro": worst_rel, "max_abs_over_ref": worst_abs, "prune_bit_exact": prune_ok,
+              "ok": not failed, "failed": failed, "tolerance": {"rel_fro": REL_FRO_TOL, "max_abs_over_ref": MAX_ABS_TOL},
+              "sample": "image 0 of every layer's output under the plan that is timed, against the CPU checker on the same input"}
+    baseline = {"value": 1.0 / t_total, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample}
+    return parity, baseline
 
 
 def main():
@@ -314,6 +331,9 @@ def main():
     ap.add_argument("--stages", type=int, default=0, help="with --variant: ring depth")
     ap.add_argument("--split", type=int, default=0, help="with --variant: the plan's split field")
     ap.add_argument("--kblk", type=int, default=0, help="with --variant: 32-column blocks per pipeline stage")
+    ap.add_argument("--loads", type=int, default=0, help="with --variant 8: 1 = im2col loads, 2 = patch loads")
+    ap.add_argument("--issuers", type=int, default=0, help="with --variant 8: MMA issuer threads")
+    ap.add_argument("--ksplit", type=int, default=0, help="with --variant 8: ranges of the reduction axis")
     ap.add_argument("--depth", type=int, default=50, choices=[18, 34, 50, 101, 152], help="ResNet depth of the conv stack")
     ap.add_argument("--net", default="resnet", choices=["resnet", "mobilenet_v2"],
                     help="mobilenet_v2: its pointwise (1x1) convolutions only, the layers the paper prunes there")
@@ -363,15 +383,15 @@ def main():
         y = torch.empty((s.batch, s.ho, s.wo, s.c_out), dtype=torch.float32, device=dev)
         if loaded is not None and s.name in loaded:
             plan = nm.nm_plan_t()
-            plan.variant, plan.bn, plan.stages, plan.split = (loaded[s.name][k] for k in ("variant", "bn", "stages", "split"))
-            plan.kblk = loaded[s.name].get("kblk", 0)
+            for k in PLAN_FIELDS:
+                setattr(plan, k, int(loaded[s.name].get(k, 0)))
             nm.nm_weights_reserve(hnd, nm.nm_plan_scratch_bytes(hnd, x.shape, s.stride, s.pad, s.dil, plan))
         elif args.variant is None:
             plan, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
         else:
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.stages, plan.split = args.variant, args.bn, args.stages, args.split
-            plan.kblk = args.kblk
+            plan.kblk, plan.loads, plan.issuers, plan.ksplit = args.kblk, args.loads, args.issuers, args.ksplit
             nm.nm_weights_reserve(hnd, nm.nm_plan_scratch_bytes(hnd, x.shape, s.stride, s.pad, s.dil, plan))
         state.append((s, hnd, x, bias, y, plan))
 
@@ -382,6 +402,10 @@ def main():
     def step():
         for s, hnd, x, bias, y, plan in state:
             nm.nm_conv2d(hnd, x, s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=y, plan=plan)
+
+    parity = baseline = None
+    if rank == 0 and world == 1 and not args.no_extras:
+        parity, baseline = parity_and_cpu_baseline(nm, state)
 
     for _ in range(args.warmup):
         step()
@@ -504,17 +528,43 @@ def main():
                 b.record()
                 b.synchronize()
                 samples.append(a.elapsed_time(b) / launches)
-            per.append(samples)
+            # the same layer on ONE buffer pair, back to back: operands that fit stay in the L2 ("warm"; context only,
+            # the roofline fractions use the cold figure)
+            warm_ms = None
+            try:
+                def warm_burst():
+                    for _k in range(launches):
+                        nm.nm_conv2d(hnd, xs[0], s.kh, s.kw, s.stride, s.pad, s.dil, bias, s.relu, y=ys[0], plan=plan)
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                wgraph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(wgraph, stream=side):
+                        warm_burst()
+                torch.cuda.current_stream().wait_stream(side)
+                wgraph.replay()
+                a, b = torch.cuda.Event(True), torch.cuda.Event(True)
+                a.record()
+                wgraph.replay()
+                b.record()
+                b.synchronize()
+                warm_ms = a.elapsed_time(b) / launches
+                del wgraph
+            except Exception:
+                torch.cuda.synchronize()
+            per.append((samples, warm_ms))
             del replay, xs, ys
         table, t_roof_sum = [], 0.0
-        for (s, hnd, x, bias, y, plan), ts in zip(state, per):
+        for (s, hnd, x, bias, y, plan), (ts, warm_ms) in zip(state, per):
             ms = statistics.median(ts)
             t_tc = useful_flops(s) / (tf32_peak * 1e12) * 1e3
             t_hbm = algorithmic_bytes(s) / (pk["hbm_gbs"] * 1e9) * 1e3
             t_roof = max(t_tc, t_hbm)
             t_roof_sum += t_roof
             table.append({"layer": s.name, "shape": f"{s.c_in}->{s.c_out} {s.kh}x{s.kw}/{s.stride} @{s.h}",
-                          "ms": round(ms, 4), "useful_tflops": round(useful_flops(s) / (ms * 1e-3) / 1e12, 2),
+                          "ms": round(ms, 4), "ms_warm": round(warm_ms, 4) if warm_ms is not None else None,
+                          "kept_columns_only": plan.variant in KEPT_ONLY_VARIANTS,
+                          "useful_tflops": round(useful_flops(s) / (ms * 1e-3) / 1e12, 2),
                           "gbs": round(algorithmic_bytes(s) / (ms * 1e-3) / 1e9, 1),
                           "bound": "tensor" if t_tc > t_hbm else "hbm", "roofline_frac": round(t_roof / ms, 3),
                           "plan": plan.as_dict()})
@@ -523,6 +573,39 @@ def main():
                                       "divided by the measured time of a step")
         out["per_layer"] = table
         out["per_layer_mode"] = per_layer_mode
+        out["per_layer_note"] = ("ms: cold (rotating buffer sets larger than twice the L2, every launch finds its operands in HBM); "
+                                 "ms_warm: the same launch repeated on one buffer pair (operands that fit stay in L2)")
+        out["layers_at_half_roofline"] = sum(1 for r in table if r["roofline_frac"] >= 0.5)
+        out["launches_kept_columns_only"] = sum(1 for r in table if r["kept_columns_only"])
+        # tile width as a tuning knob (Sec. 3.3, Sec. 4.4) on the tensor-bound layers: per candidate T the fastest plan,
+        # the fastest plan among the kernels that skip the pruned columns, and the share of the L1 mass the
+        # pruning retains (the accuracy proxy: wider tiles share a kept set among more rows and retain less)
+        if args.variant is None and not args.load_plans and not args.layer:
+            choice = []
+            for li, ((s, hnd, x, bias, y, plan), row) in enumerate(zip(state, table)):
+                if row["bound"] != "tensor" or s.n_keep == s.m_group:
+                    continue
+                w = inputs.make_weights(s, li).to(dev)
+                cands = []
+                for t in (64, 128, 256):
+                    if s.c_out % t != 0:
+                        continue
+                    h_t = nm.nm_prune(w, s.n_keep, s.m_group, t)
+                    kept, total = nm.nm_weights_retained_l1(h_t)
+                    p_all, ms_all = nm.nm_autotune(h_t, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
+                    os.environ["NM_AUTOTUNE_VARIANTS"] = ",".join(str(v) for v in KEPT_ONLY_VARIANTS)
+                    p_kept, ms_kept = nm.nm_autotune(h_t, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
+                    del os.environ["NM_AUTOTUNE_VARIANTS"]
+                    cands.append({"tile_t": t, "retained_l1": round(kept / total, 4), "ms": round(ms_all, 4),
+                                  "variant": p_all.variant, "ms_kept_columns_only": round(ms_kept, 4),
+                                  "variant_kept_columns_only": p_kept.variant})
+                    h_t.free()
+                best = min(cands, key=lambda c: c["ms"])
+                choice.append({"layer": s.name, "candidates": cands, "fastest_tile_t": best["tile_t"]})
+                del w
+            out["tile_choice"] = {"layers": choice,
+                                  "note": "single cold launches timed by nm_autotune (median of 9); the headline keeps T = "
+                                          f"{WORKLOAD['tile']} for every layer"}
         # roofline object: the kernel that takes the largest share of a step, over all its launches
         by_kernel = {}
         for (s, hnd, x, bias, y, plan), row in zip(state, table):
@@ -555,11 +638,11 @@ def main():
                     "than twice the L2)",
         }
 
-        # the same stack restricted to the kernels that gather only the retained columns (variants 1-3:
-        # Algorithm 1 proper, kept FLOPs only); the headline lets the auto-tuner also take the
+        # the same stack restricted to the kernels that contract over the retained columns only (variants
+        # 1-3 and 8: Algorithm 1 proper, kept FLOPs only); the headline lets the auto-tuner also take the
         # expanded-operand kernels, which multiply the zeros
         if args.variant is None and not args.load_plans and not args.layer:
-            os.environ["NM_AUTOTUNE_VARIANTS"] = "1,2,3"
+            os.environ["NM_AUTOTUNE_VARIANTS"] = ",".join(str(v) for v in KEPT_ONLY_VARIANTS)
             gplans = []
             for s, hnd, x, bias, y, plan in state:
                 gp, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
@@ -581,7 +664,10 @@ def main():
             g_ms = a.elapsed_time(b) / args.steps
             out["gather_only"] = {"value": args.batch / (g_ms * 1e-3), "unit": UNIT, "ms_per_step": g_ms,
                                   "useful_tflops": flops_step / (g_ms * 1e-3) / 1e12,
-                                  "note": "plans restricted to the gathering kernels (variants 1-3)"}
+                                  "variants": {str(v): sum(1 for gp in gplans if gp.variant == v) for v in KEPT_ONLY_VARIANTS},
+                                  "note": "plans restricted to the kernels that contract over the retained columns only "
+                                          "(variants 1-3 and 8: Algorithm 1 proper); the headline lets the tuner also take the "
+                                          "expanded-operand kernels, which multiply the zeros of the pruned columns"}
 
         # the same layers chained as the network's dataflow: stem -> max-pool -> residual blocks, every
         # layer reading its predecessor's output, shortcut additions fused into the last conv of a block
@@ -795,7 +881,8 @@ def main():
                       "note": "every layer's input copied from pinned host memory and every output copied back "
                               "(nm_conv2d_host per layer, three streams)"}
         del host
-        out["cpu_baseline"] = cpu_baseline()
+        out["cpu_baseline"] = baseline
+        out["parity"] = parity
 
     if rank == 0:
         if args.json_out:
@@ -805,6 +892,8 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+    if parity is not None and not parity["ok"]:
+        sys.exit(1)   # a timed plan whose output is wrong is not a result
 
 
 if __name__ == "__main__":

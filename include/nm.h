@@ -248,6 +248,10 @@ nm_status_t nm_weights_free(nm_weights_t* w);
  *   y[n][oh][ow][o] = act( bias[o] + sum_j values[o][j] *
  *                          x[n][oh*stride_h - pad_h + kh_j*dil_h][ow*stride_w - pad_w + kw_j*dil_w][c_j] )
  * with (kh_j, kw_j, c_j) decoded from indices[o / tile_t][j] and reads outside the image = 0.
+ * Non-finite activations: the kernels that contract over the retained columns only (variants 1, 2, 3, 8) never
+ * read a pruned column's activation, as Algorithm 1 does not; the expanded-operand kernels (variants 4-7)
+ * multiply it by a zero weight, so an Inf or NaN in a PRUNED column turns the outputs of that pixel into NaN there
+ * while the definition above (and variants 1, 2, 3, 8) keep them finite.  Finite inputs give the same results in all.
  * Arithmetic: operands rounded to TF32 (weights once at prune time, round-to-nearest; activations
  * round-to-nearest where they pass through registers (variants 1-3), truncated where the staged
  * slab feeds the tensor core directly (variants 4, 5, 6)), products accumulated in fp32.
@@ -314,10 +318,14 @@ nm_status_t nm_maxpool2d(const float* x, int batch, int h, int w, int c, int kh,
  * layers that would fit the cache are tuned for operands that come from HBM.  Candidates are tried
  * most promising first and a later one replaces the best so far only if it is at least 1 % faster.
  * This call allocates (the buffer above, and the split-K scratch described at nm_weights_reserve).
- * The environment variable NM_AUTOTUNE_VARIANTS (a list of variant digits such as "1,2,3") restricts the
- * search, e.g. to the kernels that skip the pruned columns.
+ * The environment variable NM_AUTOTUNE_VARIANTS (a list of variant digits such as "1,2,3,8") restricts the
+ * search, e.g. to the kernels that skip the pruned columns.  The handle is not const: the call reserves
+ * scratch memory on it.
+ * Plan cache: when the environment variable NM_PLAN_CACHE names a file, the call first looks the layer up there
+ * (key: nm_plan_key of the layer) and, if the cached plan still runs, returns it without tuning (its time is
+ * measured over a few launches); otherwise it tunes and appends the result to the file.
  */
-nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h, int wd,
+nm_status_t nm_autotune(nm_weights_t* w, const float* x, int batch, int h, int wd,
                         int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
                         const float* bias, int relu, float* y_scratch, void* cuda_stream,
                         nm_plan_t* best, float* best_ms);
@@ -347,6 +355,23 @@ nm_status_t nm_autotune_tile(const float* w_dense, int c_out, int kh, int kw, in
  * faults, traps or hangs.
  */
 nm_status_t nm_selftest_wait_expiry(const nm_weights_t* w, void* cuda_stream);
+
+/*
+ * Plan cache: a text file with one line per layer, "<key> variant bn stages split kblk loads issuers ksplit"
+ * (the analogue of keeping the profiler's choice per operator, Sec. 3.3; the last line of a key wins).
+ *   nm_plan_key           writes the key of a layer (its geometry, pattern and tile width, batch and image size,
+ *                         whether it has a bias / ReLU) into `key` (at most key_bytes, NUL-terminated);
+ *                         INVALID_ARG if the buffer is too small
+ *   nm_plan_cache_store   appends (key, plan) to the file (created if missing); CUDA is not touched
+ *   nm_plan_cache_lookup  fills *plan from the file; NM_ERR_UNSUPPORTED if the file or the key is missing
+ * A plan taken from a cache is only data: nm_conv2d checks it against the layer like any other plan, and a plan
+ * that needs scratch memory still needs nm_plan_scratch_bytes / nm_weights_reserve before its first use.
+ */
+nm_status_t nm_plan_key(int c_out, int kh, int kw, int c_in, int n_keep, int m_group, int tile_t, int batch, int h,
+                        int wd, int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w, int has_bias,
+                        int relu, char* key, size_t key_bytes);
+nm_status_t nm_plan_cache_store(const char* path, const char* key, const nm_plan_t* plan);
+nm_status_t nm_plan_cache_lookup(const char* path, const char* key, nm_plan_t* plan);
 
 const char* nm_status_string(nm_status_t s);
 /* Text of the calling thread's most recent failure ("" if none). Valid until its next failure. */

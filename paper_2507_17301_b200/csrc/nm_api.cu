@@ -486,7 +486,54 @@ nm_status_t nm_conv2d_host(const nm_weights_t* w, const float* x_host, float* x_
     return NM_OK;
 }
 
-nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h, int wd, int stride_h, int stride_w,
+nm_status_t nm_plan_key(int c_out, int kh, int kw, int c_in, int n_keep, int m_group, int tile_t, int batch, int h, int wd,
+                        int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w, int has_bias, int relu,
+                        char* key, size_t key_bytes)
+{
+    if (!key || key_bytes == 0) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_plan_key: key buffer missing");
+    const int n = std::snprintf(key, key_bytes, "co%d_k%dx%d_ci%d_nm%d:%d_t%d_b%d_hw%dx%d_s%dx%d_p%dx%d_d%dx%d_bias%d_relu%d", c_out, kh,
+                                kw, c_in, n_keep, m_group, tile_t, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                has_bias ? 1 : 0, relu ? 1 : 0);
+    if (n < 0 || static_cast<size_t>(n) >= key_bytes) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_plan_key: key buffer too small");
+    return NM_OK;
+}
+
+nm_status_t nm_plan_cache_store(const char* path, const char* key, const nm_plan_t* plan)
+{
+    if (!path || !key || !plan || !key[0] || std::strpbrk(key, " \t\n"))
+        return nmhost::fail(NM_ERR_INVALID_ARG, "nm_plan_cache_store: path, key (no blanks) and plan are required");
+    std::FILE* f = std::fopen(path, "a");
+    if (!f) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_plan_cache_store: cannot open %s", path);
+    const int n = std::fprintf(f, "%s %d %d %d %d %d %d %d %d\n", key, plan->variant, plan->bn, plan->stages, plan->split, plan->kblk,
+                               plan->loads, plan->issuers, plan->ksplit);
+    const bool ok = n > 0 && std::fclose(f) == 0;
+    if (!ok) return nmhost::fail(NM_ERR_INTERNAL, "nm_plan_cache_store: write to %s failed", path);
+    return NM_OK;
+}
+
+nm_status_t nm_plan_cache_lookup(const char* path, const char* key, nm_plan_t* plan)
+{
+    if (!path || !key || !plan) return nmhost::fail(NM_ERR_INVALID_ARG, "nm_plan_cache_lookup: path, key and plan are required");
+    std::FILE* f = std::fopen(path, "r");
+    if (!f) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_plan_cache_lookup: no cache file %s", path);
+    char line[512], k[384];
+    bool found = false;
+    nm_plan_t p;
+    while (std::fgets(line, sizeof(line), f)) {
+        std::memset(&p, 0, sizeof(p));
+        if (std::sscanf(line, "%383s %d %d %d %d %d %d %d %d", k, &p.variant, &p.bn, &p.stages, &p.split, &p.kblk, &p.loads,
+                        &p.issuers, &p.ksplit) == 9 &&
+            std::strcmp(k, key) == 0) {
+            *plan = p;      // the last line of a key wins
+            found = true;
+        }
+    }
+    std::fclose(f);
+    if (!found) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_plan_cache_lookup: no entry for %s", key);
+    return NM_OK;
+}
+
+nm_status_t nm_autotune(nm_weights_t* w, const float* x, int batch, int h, int wd, int stride_h, int stride_w,
                         int pad_h, int pad_w, int dil_h, int dil_w, const float* bias, int relu, float* y_scratch,
                         void* cuda_stream, nm_plan_t* best, float* best_ms)
 {
@@ -500,7 +547,7 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
     // split over several CTAs; the partial sums need scratch memory, which belongs to the handle
     // and is reserved here (nm_conv2d itself never allocates).
     {
-        nm_weights* hw = const_cast<nm_weights*>(w);
+        nm_weights* hw = w;
         int n_sm = 148, dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         const long long pix_blocks = (p.pixels + 127) / 128;
@@ -529,6 +576,39 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
     }
     constexpr int kWarm = 2, kReps = 9;
     float best_t = -1.f;
+    // plan cache: a cached plan that still runs on this layer is returned with its time over three launches
+    char key[384] = "";
+    const char* cache = std::getenv("NM_PLAN_CACHE");
+    if (cache && cache[0] &&
+        nm_plan_key(w->c_out, w->kh, w->kw, w->c_in, w->n_keep, w->m_group, w->tile_t, batch, h, wd, stride_h, stride_w, pad_h,
+                    pad_w, dil_h, dil_w, bias != nullptr, relu, key, sizeof(key)) == NM_OK) {
+        nm_plan_t cached;
+        if (nm_plan_cache_lookup(cache, key, &cached) == NM_OK) {
+            size_t need = 0;
+            if (nm_plan_scratch_bytes(w, batch, h, wd, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, &cached, &need) == NM_OK &&
+                (need <= w->splitk_bytes || nm_weights_reserve(w, need) == NM_OK)) {
+                p.splitk = w->splitk;
+                p.splitk_bytes = w->splitk_bytes;
+                bool ok = run_plan(p, &cached, st) == NM_OK && cudaStreamSynchronize(st) == cudaSuccess;
+                float ms = 0.f;
+                if (ok) {
+                    cudaEventRecord(e0, st);
+                    for (int i = 0; i < 3 && ok; ++i) ok = run_plan(p, &cached, st) == NM_OK;
+                    cudaEventRecord(e1, st);
+                    ok = ok && cudaEventSynchronize(e1) == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
+                }
+                if (ok) {
+                    *best = cached;
+                    if (best_ms) *best_ms = ms / 3.f;
+                    if (flush) cudaFree(flush);
+                    cudaEventDestroy(e0);
+                    cudaEventDestroy(e1);
+                    return nm_weights_check(w, cuda_stream);
+                }
+            }
+            (void)cudaGetLastError();
+        }
+    }
     for (const nm_plan_t& cand : candidate_plans(w, p)) {
         bool ok = true;
         for (int i = 0; i < kWarm && ok; ++i) ok = run_plan(p, &cand, st) == NM_OK;
@@ -557,6 +637,7 @@ nm_status_t nm_autotune(const nm_weights_t* w, const float* x, int batch, int h,
     cudaEventDestroy(e1);
     if (best_t < 0.f) return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_autotune: no candidate plan ran");
     if (best_ms) *best_ms = best_t;
+    if (cache && cache[0] && key[0]) (void)nm_plan_cache_store(cache, key, best);
     return nm_weights_check(w, cuda_stream);
 }
 

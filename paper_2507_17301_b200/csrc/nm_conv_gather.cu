@@ -88,8 +88,12 @@ __global__ void __launch_bounds__(128) k_conv_gather(const ConvParams p, const i
             const int ih = s_row_ih0[row] + dh, iw = s_row_iw0[row] + dw;
             float v = 0.f;
             if (tap_ok && n >= 0 && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w)
+                // self-checking build: the tap table may only name taps and channels of this layer
+                NM_CHECKED(c < p.c_in && static_cast<int>(tap >> 24) < p.kh && static_cast<int>((tap >> 16) & 0xFFu) < p.kw && n < p.batch,
+                           p.status, 101, tap)
                 v = __ldg(p.x + ((static_cast<size_t>(n) * p.h + ih) * p.w + iw) * p.c_in + c);
             const uint32_t dst = a_base + row * 128 + ((((lane >> 2) ^ (row & 7))) << 4) + ((lane & 3) << 2);
+            NM_CHECKED(dst >= a_base && dst + 4 <= a_base + A_BYTES, p.status, 102, dst - a_base)
             asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(to_tf32(v)) : "memory");
         }
         // weight chunk [umma_n rows x 32 columns]; rows past the tile or past c_out are zero

@@ -225,7 +225,9 @@ k_conv_slab(const ConvParams p, const SlabCfg cfg, const __grid_constant__ CUten
                     const uint32_t rel = (relw[j >> 2] >> ((j & 3) * 8)) & 0xFFu;
                     // sub-tile (rel / 32), 16-byte piece ((rel / 4) % 8) ^ (row % 8), word rel % 4
                     const uint32_t u = ((rel & 31u) << 2) + ((rel >> 5) * SUB_BYTES);
-                    float f;
+                    float f = 0.f;
+                    // self-checking build: a kept-column offset must lie inside the chunk's source columns
+                    NM_CHECKED(rel < static_cast<uint32_t>(p.v2_s), p.status, 201, rel)
                     asm volatile("ld.shared.f32 %0, [%1];" : "=f"(f) : "r"(slab_row + (u ^ rx4)));
                     v[j] = __float_as_uint(to_tf32(f));
                 }

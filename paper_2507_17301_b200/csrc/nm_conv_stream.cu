@@ -357,8 +357,10 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
 #pragma unroll
                 for (int i = 0; i < P::LW; ++i) {
                     const int ci = ci0 + i;
-                    L[i] = live ? lds128(slab + (ci >> 3) * SUB_BYTES + row * 128 + ((static_cast<uint32_t>(ci & 7) ^ rx) << 4))
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    L[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    // self-checking build: the row's pieces lie inside this stage's slab
+                    NM_CHECKED((ci >> 3) < P::SEGS && slab + (ci >> 3) * SUB_BYTES + row * 128 + 128 <= relbuf, p.status, 301, ci)
+                    if (live) L[i] = lds128(slab + (ci >> 3) * SUB_BYTES + row * 128 + ((static_cast<uint32_t>(ci & 7) ^ rx) << 4));
                 }
                 const uint32_t a_set = tmem + lane_addr + A_COL0 + set * cfg.set_cols + wg * P::KW;
                 for (int t = 0; t < g; ++t) {
@@ -376,6 +378,9 @@ k_conv_stream(const ConvParams p, const StreamCfg cfg, const __grid_constant__ C
                             f = (j & 3) == 0 ? l4.x : (j & 3) == 1 ? l4.y : (j & 3) == 2 ? l4.z : l4.w;
                         } else {
                             const uint32_t r = (sel[j >> 2] >> (8 * (j & 3))) & static_cast<uint32_t>(MG - 1);
+                            f = 0.f;
+                            // self-checking build: a kept-column offset, taken whole, lies inside the chunk's source columns
+                            NM_CHECKED(((sel[j >> 2] >> (8 * (j & 3))) & 0xFFu) < static_cast<uint32_t>(P::S), p.status, 302, sel[j >> 2])
                             f = pick<MG>(&L[(j / NK) * (MG / 4)], r);
                         }
                         v[j] = round_tf32_bits(f);   // a half that was not loaded holds zeros: 0x1000 is below TF32's last bit

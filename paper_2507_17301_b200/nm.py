@@ -78,6 +78,12 @@ def _load():
     for name in ("nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
                  "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile"):
         getattr(lib, name).restype = ctypes.c_int
+    lib.nm_plan_key.argtypes = [i] * 18 + [ctypes.c_char_p, ctypes.c_size_t]
+    lib.nm_plan_key.restype = ctypes.c_int
+    lib.nm_plan_cache_store.argtypes = [ctypes.c_char_p, ctypes.c_char_p, pp]
+    lib.nm_plan_cache_store.restype = ctypes.c_int
+    lib.nm_plan_cache_lookup.argtypes = [ctypes.c_char_p, ctypes.c_char_p, pp]
+    lib.nm_plan_cache_lookup.restype = ctypes.c_int
     lib.nm_status_string.argtypes = [ctypes.c_int]
     lib.nm_status_string.restype = ctypes.c_char_p
     lib.nm_last_error.argtypes = []
@@ -89,7 +95,7 @@ def _load():
 
 _lib = _load()
 
-EXPORTS = ("nm_selftest_wait_expiry", "nm_maxpool2d", "nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
+EXPORTS = ("nm_plan_key", "nm_plan_cache_store", "nm_plan_cache_lookup", "nm_selftest_wait_expiry", "nm_maxpool2d", "nm_weights_retained_l1", "nm_conv2d_res", "nm_plan_scratch_bytes", "nm_weights_reserve", "nm_prune", "nm_prune_noalloc", "nm_weights_dims", "nm_weights_export", "nm_weights_import", "nm_weights_check",
            "nm_weights_free", "nm_conv2d", "nm_conv2d_host", "nm_autotune", "nm_autotune_tile",
            "nm_status_string", "nm_last_error", "nm_launch_count")
 
@@ -241,6 +247,31 @@ def nm_weights_retained_l1(w: Weights):
     kept, total = ctypes.c_double(), ctypes.c_double()
     _check(_lib.nm_weights_retained_l1(w.handle, ctypes.byref(kept), ctypes.byref(total)))
     return float(kept.value), float(total.value)
+
+
+def nm_plan_key(c_out, kh, kw, c_in, n_keep, m_group, tile_t, x_shape, stride=1, pad=0, dil=1, has_bias=True,
+                relu=False) -> str:
+    """Key of a layer in the plan cache file (geometry, pattern, tile width, batch and image size, bias / ReLU)."""
+    stride, pad, dil = _pair(stride), _pair(pad), _pair(dil)
+    b, h, wd, _ = x_shape
+    buf = ctypes.create_string_buffer(384)
+    _check(_lib.nm_plan_key(c_out, kh, kw, c_in, n_keep, m_group, tile_t, b, h, wd, stride[0], stride[1], pad[0], pad[1],
+                            dil[0], dil[1], int(bool(has_bias)), int(bool(relu)), buf, len(buf)))
+    return buf.value.decode()
+
+
+def nm_plan_cache_store(path: str, key: str, plan: nm_plan_t) -> None:
+    _check(_lib.nm_plan_cache_store(path.encode(), key.encode(), ctypes.byref(plan)))
+
+
+def nm_plan_cache_lookup(path: str, key: str):
+    """The cached plan of `key`, or None when the file or the key is missing."""
+    plan = nm_plan_t()
+    status = _lib.nm_plan_cache_lookup(path.encode(), key.encode(), ctypes.byref(plan))
+    if status == NM_ERR_UNSUPPORTED:
+        return None
+    _check(status)
+    return plan
 
 
 def nm_selftest_wait_expiry(w: Weights):

@@ -75,3 +75,28 @@ def test_product_path_does_not_touch_the_oracle():
                 text = open(os.path.join(dirpath, f)).read()
                 for needle in ("import oracle", "from oracle", "nm_oracle", "oracle/"):
                     assert needle not in text, f"{f} reaches for the CPU oracle ({needle})"
+
+
+def test_plan_cache_file_round_trip(lib_path, tmp_path):
+    """The plan cache is host-side text: store, look up, last line of a key wins, missing entries are reported."""
+    from paper_2507_17301_b200 import nm
+    path = str(tmp_path / "plans.txt")
+    key = nm.nm_plan_key(256, 3, 3, 256, 2, 4, 64, (64, 14, 14, 256), 1, 1, 1, True, True)
+    other = nm.nm_plan_key(256, 3, 3, 256, 2, 4, 128, (64, 14, 14, 256), 1, 1, 1, True, True)
+    assert key != other and " " not in key and "t64" in key and "t128" in other
+    assert nm.nm_plan_cache_lookup(path, key) is None                      # no file yet
+    p = nm.nm_plan_t()
+    p.variant, p.bn, p.stages, p.split, p.kblk, p.loads, p.issuers, p.ksplit = 8, 256, 2, 0, 0, 2, 4, 3
+    nm.nm_plan_cache_store(path, key, p)
+    assert nm.nm_plan_cache_lookup(path, other) is None                    # another layer
+    got = nm.nm_plan_cache_lookup(path, key)
+    assert got.as_dict() == p.as_dict()
+    p.variant, p.bn, p.ksplit = 4, 128, 0
+    nm.nm_plan_cache_store(path, key, p)                                   # a newer entry replaces the older one
+    assert nm.nm_plan_cache_lookup(path, key).as_dict() == p.as_dict()
+    assert len(open(path).read().splitlines()) == 2
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_plan_cache_store(path, "a key with blanks", p)
+    assert e.value.status == nm.NM_ERR_INVALID_ARG
+    buf = ctypes.create_string_buffer(8)                                   # a key buffer that is too small
+    assert nm._lib.nm_plan_key(*([1] * 18), buf, len(buf)) == nm.NM_ERR_INVALID_ARG

@@ -457,3 +457,71 @@ def test_autotune_returns_a_working_plan(nm):
     tile, plan, ms = nm.nm_autotune_tile(w.cuda(), s.n_keep, s.m_group, [16, 32], x.cuda(), s.stride, s.pad, s.dil,
                                          b.cuda(), s.relu)
     assert tile in (16, 32) and ms > 0
+
+
+def test_autotune_uses_the_plan_cache(nm, tmp_path, monkeypatch):
+    """With NM_PLAN_CACHE set, nm_autotune stores what it found and the next call on the same layer returns that
+    plan without tuning; a cached plan the layer does not admit is ignored and replaced."""
+    s = ConvShape("cache_3x3", 2, 16, 16, 64, 64, 3, 3, 1, 1, 1, 2, 4, 32)
+    w, x, b = tensors_for(s)
+    vr, ir, yr = oracle_layer(s, w, x, b)
+    path = str(tmp_path / "plans.txt")
+    monkeypatch.setenv("NM_PLAN_CACHE", path)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    xd, bd = x.cuda(), b.cuda()
+    plan1, ms1 = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)
+    key = nm.nm_plan_key(s.c_out, s.kh, s.kw, s.c_in, s.n_keep, s.m_group, s.tile_t, xd.shape, s.stride, s.pad, s.dil, True, s.relu)
+    assert nm.nm_plan_cache_lookup(path, key).as_dict() == plan1.as_dict()
+    forced = nm.nm_plan_t()
+    forced.variant = 1                                  # the slowest kernel: tuning would never pick it here
+    nm.nm_plan_cache_store(path, key, forced)
+    plan2, ms2 = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)
+    assert plan2.variant == 1 and ms2 > 0
+    y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan2)
+    torch.cuda.synchronize()
+    assert_conv_close(y.cpu().numpy(), yr)
+    bad = nm.nm_plan_t()
+    bad.variant, bad.bn = 4, 96                         # 96 channels per CTA do not divide 64: not admissible
+    nm.nm_plan_cache_store(path, key, bad)
+    plan3, _ = nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, s.relu, kh=s.kh, kw=s.kw)
+    assert plan3.as_dict() != bad.as_dict()
+    assert nm.nm_plan_cache_lookup(path, key).as_dict() == plan3.as_dict()
+
+
+def test_balanced_plan_beside_a_busy_stream(nm):
+    """A balanced plan's CTAs wait (with a bound) for flags raised by other CTAs of the same launch, which assumes
+    that all of them are resident.  With another stream keeping SMs busy the launch must still either finish with
+    the right result or report NM_ERR_TIMEOUT through the status word: never hang, never return wrong numbers."""
+    s = BALANCED[0]
+    w, x, b = tensors_for(s, True)
+    vr, ir, yr = oracle_layer(s, w, x, b)
+    hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    other = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
+    xd, bd = x.cuda(), b.cuda()
+    plan = nm.nm_plan_t()
+    plan.variant, plan.bn, plan.split = 4, 64, -1
+    nm.nm_weights_reserve(hnd, nm.nm_plan_scratch_bytes(hnd, xd.shape, s.stride, s.pad, s.dil, plan))
+    busy = torch.cuda.Stream()
+    y_other = torch.empty((s.batch, s.ho, s.wo, s.c_out), device="cuda")
+    torch.cuda.synchronize()
+    outcomes = set()
+    for _ in range(5):
+        with torch.cuda.stream(busy):                   # a queue of persistent kernels on the other stream
+            for _k in range(20):
+                nm.nm_conv2d(other, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, y=y_other)
+        y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
+        try:
+            nm.nm_weights_check(hnd)
+            torch.cuda.synchronize()
+            assert np.array_equal(y.cpu().numpy(), yr)
+            outcomes.add("ok")
+        except nm.NmError as e:
+            assert e.status == nm.NM_ERR_TIMEOUT
+            outcomes.add("timeout")
+        torch.cuda.synchronize()
+    assert outcomes <= {"ok", "timeout"} and outcomes
+    nm.nm_weights_check(other)
+    y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)   # alone again: must be right
+    nm.nm_weights_check(hnd)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy(), yr)
