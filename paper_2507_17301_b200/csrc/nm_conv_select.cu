@@ -97,31 +97,6 @@ __device__ __forceinline__ void lds128(uint32_t addr, uint32_t* dst)
 {
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(dst[0]), "=r"(dst[1]), "=r"(dst[2]), "=r"(dst[3]) : "r"(addr));
 }
-// `n` consecutive 32-bit words of shared memory (n a compile-time constant, addr aligned to `align` bytes).
-template <int N, int ALIGN>
-__device__ __forceinline__ void lds_words(uint32_t addr, uint32_t* dst)
-{
-    if constexpr (ALIGN % 16 == 0 && N % 4 == 0) {
-#pragma unroll
-        for (int i = 0; i < N / 4; ++i) lds128(addr + 16 * i, dst + 4 * i);
-    } else if constexpr (ALIGN % 8 == 0 && N % 2 == 0) {
-#pragma unroll
-        for (int i = 0; i < N / 2; ++i)
-            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(dst[2 * i]), "=r"(dst[2 * i + 1]) : "r"(addr + 8 * i));
-    } else {
-#pragma unroll
-        for (int i = 0; i < N; ++i) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(dst[i]) : "r"(addr + 4 * i));
-    }
-}
-// Byte `k` of `w` (0x80 = set, 0x00 = clear) widened to a 32-bit mask of all ones / all zeros: one byte permute
-// whose four selectors replicate the sign bit of the chosen byte.
-template <int K>
-__device__ __forceinline__ uint32_t mask_of_byte(uint32_t w)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(d) : "r"(w), "n"(0x8888 | (0x1111 * K)));
-    return d;
-}
 // m ? a : b, bit by bit (m is all ones or all zeros)
 __device__ __forceinline__ uint32_t bsel(uint32_t m, uint32_t a, uint32_t b)
 {
@@ -157,9 +132,9 @@ struct Pattern {
     static constexpr int GW = GROUPS / 2;                    // groups per compactor half
     static constexpr int KW = GW * NK;                       // kept columns per compactor half
     static constexpr int LW = S / 8;                         // 16-byte pieces of a row per compactor half
-    static constexpr int MW = GROUPS * NK * D;               // select masks (one byte each) per tile and chunk
-    static constexpr int HW = MW / 2;                        // ... per half of the chunk
-    static constexpr int MWP = (MW + 15) / 16 * 16;          // bytes a tile's masks of one chunk occupy (bulk copies move 16-byte units)
+    static constexpr int MW = GROUPS * NK * D;               // select masks (32-bit words) per tile and chunk
+    static constexpr int HW = MW / 2;                        // ... per half of the chunk (a multiple of 4 for every pattern)
+    static constexpr int MWP = MW * 4;                       // bytes a tile's masks of one chunk occupy
 };
 
 struct Item {
@@ -540,15 +515,18 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                             pre_w = mbar_test_wait(smem_u32(&s_wfull[nw.s]), nw.parity);
                             pre_a = mbar_test_wait(smem_u32(&s_wfree[no.s]), no.parity);
                         }
-                        const uint32_t mbase = wst + cfg.w_bytes + half * P::HW;
+                        const uint32_t mbase = wst + cfg.w_bytes + half * (P::HW * 4);
                         for (int tile = 0; tile < g; ++tile) {
-                            constexpr int MWORDS = (P::HW + 3) / 4;
-                            constexpr int MALIGN = P::HW % 16 == 0 ? 16 : P::HW % 8 == 0 ? 8 : 4;
-                            uint32_t M[MWORDS];   // this half's select masks of the tile, one byte each
+                            // this half's select masks of the tile: full-width words (a byte per mask widened by a byte
+                            // permute moves less through shared memory but doubles the work of the ALU pipe, which
+                            // executes logic operations at half rate and is the busier of the two with several tiles)
+                            uint32_t M[P::HW];
 #pragma unroll
-                            for (int i = 0; i < MWORDS; ++i) M[i] = 0u;
-                            NM_CHECKED(mbase + tile * P::MWP + MWORDS * 4 <= ring_end && mbase >= w_ring && (mbase & 3u) == 0u, p.status, 803, mbase)
-                            lds_words<MWORDS, MALIGN>(mbase + tile * P::MWP, M);
+                            for (int i = 0; i < P::HW / 4; ++i) {
+                                M[4 * i] = M[4 * i + 1] = M[4 * i + 2] = M[4 * i + 3] = 0u;
+                                NM_CHECKED(mbase + tile * P::MWP + i * 16 + 16 <= ring_end && mbase >= w_ring && (mbase & 15u) == 0u, p.status, 803, mbase)
+                                lds128(mbase + tile * P::MWP + i * 16, M + 4 * i);
+                            }
                             uint32_t v[P::KW];
 #pragma unroll
                             for (int gi = 0; gi < P::GW; ++gi) {
@@ -556,17 +534,7 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                                 for (int j = 0; j < NK; ++j) {
                                     uint32_t r = x[gi * MG + j + P::D];
 #pragma unroll
-                                    for (int i = P::D - 1; i >= 0; --i) {
-                                        const int mi = (gi * NK + j) * P::D + i;
-                                        uint32_t m;
-                                        switch (mi & 3) {
-                                            case 0: m = mask_of_byte<0>(M[mi >> 2]); break;
-                                            case 1: m = mask_of_byte<1>(M[mi >> 2]); break;
-                                            case 2: m = mask_of_byte<2>(M[mi >> 2]); break;
-                                            default: m = mask_of_byte<3>(M[mi >> 2]); break;
-                                        }
-                                        r = bsel(m, x[gi * MG + j + i], r);
-                                    }
+                                    for (int i = P::D - 1; i >= 0; --i) r = bsel(M[(gi * NK + j) * P::D + i], x[gi * MG + j + i], r);
                                     v[gi * NK + j] = r;
                                 }
                             }
@@ -723,7 +691,7 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     if (cfg->n_work >= (1ll << 31)) return false;
     cfg->alias_staging = cfg->n_work <= sm_count();
     // alignment slack, static shared, and the output staging unless it can lie over the ring
-    const int budget = 227 * 1024 - 1024 - 2048 - (cfg->alias_staging ? 0 : STAGING_BYTES);
+    const int budget = 227 * 1024 - 1024 - 4096 - (cfg->alias_staging ? 0 : STAGING_BYTES);   // static: barriers, 1 KB of zero rows and their alignment
     const bool paired = cfg->taps == 1;
     int n_p = 2;
     if (plan && plan->stages > 0) n_p = plan->stages;
@@ -809,8 +777,8 @@ __global__ void k_build_w3(const float* __restrict__ values, const uint16_t* __r
         nmk::to_tf32(values[static_cast<size_t>(o) * kk + j]);
 }
 
-// Select masks: for retained column j (the jn-th of its group, at position pos in the group) the D = M - N bytes
-// m[i] = 0x80 iff pos == jn + i, i < D (all zero: the column is the last candidate, jn + D); `mw` bytes per tile and chunk.
+// Select masks: for retained column j (the jn-th of its group, at position pos in the group) the D = M - N words
+// m[i] = all ones iff pos == jn + i, i < D (all zero: the column is the last candidate, jn + D); `mw` bytes per tile and chunk.
 __global__ void k_build_sel3(const uint16_t* __restrict__ indices, int n_tiles, int kk, int n_keep, int m_group,
                              int s_cols, int kc, int mw, uint8_t* __restrict__ sel3)
 {
@@ -823,8 +791,8 @@ __global__ void k_build_sel3(const uint16_t* __restrict__ indices, int n_tiles, 
     const int jj = j - chunk * kc;           // slot within the chunk = group-in-chunk * N + jn
     const int jn = jj % n_keep;
     const int pos = col % m_group;
-    uint8_t* m = sel3 + (static_cast<size_t>(chunk) * n_tiles + r) * mw + static_cast<size_t>(jj) * d;
-    for (int i = 0; i < d; ++i) m[i] = (pos == jn + i) ? 0x80u : 0u;
+    uint32_t* m = reinterpret_cast<uint32_t*>(sel3 + (static_cast<size_t>(chunk) * n_tiles + r) * mw) + static_cast<size_t>(jj) * d;
+    for (int i = 0; i < d; ++i) m[i] = (pos == jn + i) ? 0xFFFFFFFFu : 0u;
 }
 
 }  // namespace

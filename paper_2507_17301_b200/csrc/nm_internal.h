@@ -36,7 +36,7 @@ struct nm_weights {
     // Select layout (variant 8): chunks of sel_s source columns of which every tile keeps sel_kc; NULL when the
     // pattern or the shape rules the variant out.
     float* w3;           // [k / sel_s][c_out][32] TF32, rows swizzled (see k_build_w3)
-    uint8_t* sel3;       // [k / sel_s][n_tiles][sel_mw] select masks, one byte each (see k_build_sel3)
+    uint8_t* sel3;       // [k / sel_s][n_tiles][sel_mw bytes] select masks, 32-bit words (see k_build_sel3)
     int sel_s, sel_kc, sel_mw;
 };
 

@@ -1,0 +1,211 @@
+// Hardware rates that shaped the convolution kernels, measured in isolation on one GPU (every SM runs the same loop):
+//
+//   select   a compactor's inner loop: 128 pixel rows x 64 source columns read from a 128-byte-swizzled slab with
+//            16-byte loads, the 2:4 retained columns of `g` tiles picked with bitwise selects, results stored to tensor
+//            memory.  Modes: copy (no selection: the cost of reading the slab), word masks (one 32-bit mask per select,
+//            loaded from shared memory), byte masks (one byte per select, widened with a byte permute).
+//   mma      TF32 tcgen05.mma of shape 128 x N x 8 issued back to back by 1, 2 or 4 threads (each with accumulator
+//            columns of its own), A from tensor memory (TS) or from shared memory (SS).
+//
+// Prints cycles per unit of work from clock64 and from CUDA events.  Nothing here is used by the library.
+#include <cstdio>
+#include <cstdlib>
+#include <cuda_runtime.h>
+
+#include "../csrc/nm_ptx.cuh"
+using namespace nmk;
+
+#define CK(x)                                                                                  \
+    do {                                                                                       \
+        cudaError_t e = (x);                                                                   \
+        if (e != cudaSuccess) {                                                                \
+            std::printf("CUDA error %s at line %d\n", cudaGetErrorString(e), __LINE__);        \
+            std::exit(1);                                                                      \
+        }                                                                                      \
+    } while (0)
+
+__device__ __forceinline__ void lds128(uint32_t a, uint32_t* d)
+{
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a));
+}
+__device__ __forceinline__ uint32_t bsel(uint32_t m, uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(d) : "r"(m), "r"(a), "r"(b));
+    return d;
+}
+template <int K>
+__device__ __forceinline__ uint32_t mask_of_byte(uint32_t w)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(d) : "r"(w), "n"(0x8888 | (0x1111 * K)));
+    return d;
+}
+
+// MODE 0: copy, 1: word masks, 2: byte masks.  `warps` compactor warps (8 or 16), two per TMEM lane quadrant and half.
+template <int MODE>
+__global__ void __launch_bounds__(512, 1) k_select(int iters, int g, int warps, long long* cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t slab = base, masks = base + 32768;   // 2 x 16 KB slab, then g x 2 halves x 128 bytes of masks
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int i = tid; i < 8192 + 1024; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw)[i] = (i * 2654435761u) >> 3;
+    if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const long long t0 = clock64();
+    if (warp < warps) {
+        const int q = warp & 3, half = (warp >> 2) & 1, row = q * 32 + lane;
+        const uint32_t rx = row & 7, lane_addr = static_cast<uint32_t>(q * 32) << 16;
+        for (int it = 0; it < iters; ++it) {
+            uint32_t x[32];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) lds128(slab + half * 16384 + row * 128 + ((static_cast<uint32_t>(i) ^ rx) << 4), x + 4 * i);
+            for (int t = 0; t < g; ++t) {
+                uint32_t v[16];
+                const uint32_t mb = masks + (t * 2 + half) * 128;
+                if (MODE == 1) {
+                    uint32_t m[32];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) lds128(mb + 16 * i, m + 4 * i);
+#pragma unroll
+                    for (int gi = 0; gi < 8; ++gi) {
+                        v[2 * gi] = bsel(m[4 * gi], x[4 * gi], bsel(m[4 * gi + 1], x[4 * gi + 1], x[4 * gi + 2]));
+                        v[2 * gi + 1] = bsel(m[4 * gi + 2], x[4 * gi + 1], bsel(m[4 * gi + 3], x[4 * gi + 2], x[4 * gi + 3]));
+                    }
+                } else if (MODE == 2) {
+                    uint32_t m[8];
+                    lds128(mb, m);
+                    lds128(mb + 16, m + 4);
+#pragma unroll
+                    for (int gi = 0; gi < 8; ++gi) {
+                        v[2 * gi] = bsel(mask_of_byte<0>(m[gi]), x[4 * gi], bsel(mask_of_byte<1>(m[gi]), x[4 * gi + 1], x[4 * gi + 2]));
+                        v[2 * gi + 1] =
+                            bsel(mask_of_byte<2>(m[gi]), x[4 * gi + 1], bsel(mask_of_byte<3>(m[gi]), x[4 * gi + 2], x[4 * gi + 3]));
+                    }
+                } else {
+#pragma unroll
+                    for (int gi = 0; gi < 8; ++gi) { v[2 * gi] = x[4 * gi]; v[2 * gi + 1] = x[4 * gi + 1]; }
+                }
+                tmem_st16(tmem + lane_addr + 256 + ((it & 1) * 4 + t) * 32 + half * 16, v);
+            }
+            tmem_st_wait();
+        }
+    }
+    __syncthreads();
+    if (tid == 0) cycles[blockIdx.x] = clock64() - t0;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// `issuers` threads (lane 0 of warps 0 ..) each issue `count` MMAs 128 x n x 8 into accumulator columns of their own.
+__global__ void __launch_bounds__(256, 1) k_mma(int count, int n, int issuers, int ss, long long* cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem;
+    __shared__ uint64_t s_done[4];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int i = tid; i < 16384; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw)[i] = 0;
+    if (warp == 7) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (tid == 0) {
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&s_done[i]), 1);
+        mbar_fence_init();
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const long long t0 = clock64();
+    if (warp < issuers && lane == 0) {
+        const uint32_t idesc = umma_idesc_tf32(128, n);
+        const uint64_t bdesc = umma_desc_k_sw128(base, 1024), adesc = umma_desc_k_sw128(base + 32768, 1024);
+        const uint32_t acc = tmem + warp * (256 / issuers);   // 256 / issuers >= n
+        for (int i = 0; i < count; ++i) {
+            if (ss) umma_tf32_ss(acc, adesc + 2 * (i & 3), bdesc + 2 * (i & 3), idesc, 1u);
+            else umma_tf32_ts(acc, tmem + 256 + (i & 7) * 8, bdesc + 2 * (i & 3), idesc, 1u);
+        }
+        umma_commit(smem_u32(&s_done[warp]));
+        if (!mbar_wait(smem_u32(&s_done[warp]), 0)) std::printf("wait expired\n");
+    }
+    __syncthreads();
+    if (tid == 0) cycles[blockIdx.x] = clock64() - t0;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 7) tmem_dealloc(tmem, 512);
+}
+
+template <typename F>
+float best_ms(F f)
+{
+    cudaEvent_t a, b;
+    CK(cudaEventCreate(&a));
+    CK(cudaEventCreate(&b));
+    f();
+    CK(cudaDeviceSynchronize());
+    float best = 1e9f;
+    for (int i = 0; i < 3; ++i) {
+        CK(cudaEventRecord(a));
+        f();
+        CK(cudaEventRecord(b));
+        CK(cudaEventSynchronize(b));
+        float ms;
+        CK(cudaEventElapsedTime(&ms, a, b));
+        best = ms < best ? ms : best;
+    }
+    return best;
+}
+
+int main()
+{
+    int sms = 0;
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0));
+    long long* cyc;
+    CK(cudaMalloc(&cyc, sms * sizeof(long long)));
+    const size_t smem = 100 * 1024;
+    CK(cudaFuncSetAttribute(k_select<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    CK(cudaFuncSetAttribute(k_select<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    CK(cudaFuncSetAttribute(k_select<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    CK(cudaFuncSetAttribute(k_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    long long h = 0;
+    const char* mode_name[3] = {"copy", "word masks", "byte masks"};
+    const int iters = 4000;
+    for (int warps : {8, 16}) {
+        for (int g : {1, 2, 4}) {
+            for (int mode = 0; mode < 3; ++mode) {
+                auto run = [&] {
+                    if (mode == 0) k_select<0><<<sms, 512, smem>>>(iters, g, warps, cyc);
+                    if (mode == 1) k_select<1><<<sms, 512, smem>>>(iters, g, warps, cyc);
+                    if (mode == 2) k_select<2><<<sms, 512, smem>>>(iters, g, warps, cyc);
+                };
+                const float ms = best_ms(run);
+                CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+                const double chunks = static_cast<double>(iters) * (warps / 8);
+                std::printf("select  %-10s tiles=%d warps=%2d : %6.0f cycles per chunk of 128 rows x 64 source columns (%.1f ns)\n",
+                            mode_name[mode], g, warps, static_cast<double>(h) / chunks, ms * 1e6 / chunks);
+            }
+        }
+    }
+    for (int ss : {0, 1}) {
+        for (int n : {64, 128, 256}) {
+            for (int issuers : {1, 2, 4}) {
+                if (256 / issuers < n) continue;
+                const int count = 8192;
+                const float ms = best_ms([&] { k_mma<<<sms, 256, smem>>>(count, n, issuers, ss, cyc); });
+                CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+                const double total = static_cast<double>(count) * issuers;
+                std::printf("mma     %s N=%3d issuers=%d : %6.1f cycles per MMA, %6.1f ns, %5.0f TFLOP/s over %d SMs\n", ss ? "SS" : "TS", n,
+                            issuers, static_cast<double>(h) / total, ms * 1e6 / total,
+                            sms * total * 128.0 * n * 8 * 2 / (ms * 1e-3) / 1e12, sms);
+            }
+        }
+    }
+    CK(cudaFree(cyc));
+    return 0;
+}
