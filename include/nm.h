@@ -115,7 +115,8 @@ typedef struct {
     int split;
     int kblk;
     int loads;    /* variant 8: 0 = the library's choice, 1 = im2col loads, 2 = patch loads */
-    int issuers;  /* variant 8: MMA issuer threads, 1-4 and at most the work item's MMA units (0 = as many as possible) */
+    int issuers;  /* MMA issuer threads: variant 8: 1-4 and at most the work item's MMA units (0 = as many as possible);
+                     variant 4: 1 or 2, each with half of the item's channels (0 = 1) */
     int ksplit;   /* variant 8: ranges the reduction axis is split into, 1-8 (0 = 1); more than one needs scratch */
     int reserved[8];
 } nm_plan_t;

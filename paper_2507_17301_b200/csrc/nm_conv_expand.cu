@@ -59,6 +59,7 @@ struct ExpandCfg {
     int wres_bytes;   // bytes of the resident slice: all 32-column blocks of bn rows
     int n_sub;        // pipeline stages one work item reduces over: (K / 32) / ksplit / kblk
     int kblk;         // 32-column blocks per stage (1 or 2): one barrier round trip then covers kblk * 4 MMAs
+    int n_iss;        // MMA issuer threads (1 or 2): each owns bn / n_iss accumulator columns and weight rows
     int sub_bytes;    // bytes of one 32-column block inside a stage: activations (+ streamed weights)
     int ksplit;       // K splits (1 = none): a work item covers one of them and stores raw partial sums
     int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
@@ -153,10 +154,10 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     if (tid == 0) {
         for (int i = 0; i < NSTAGE_MAX; ++i) {
             mbar_init(smem_u32(&s_full[i]), 1);   // producer's expect-tx arrival
-            mbar_init(smem_u32(&s_free[i]), 1);   // MMA commit
+            mbar_init(smem_u32(&s_free[i]), cfg.n_iss);   // MMA commits
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&s_accfull[i]), 1);   // MMA commit
+            mbar_init(smem_u32(&s_accfull[i]), cfg.n_iss);   // MMA commits
             mbar_init(smem_u32(&s_accfree[i]), 8);   // epilogue warps
         }
         mbar_init(smem_u32(&s_wres), 1);
@@ -257,10 +258,17 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                 }
             }
         }
-    } else if (warp == 1) {
-        // =========================== MMA issuer ===========================
-        if (lane == 0) {
-            const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
+    } else if (warp == 1 || warp == 3) {
+        // =========================== MMA issuers ===========================
+        // A thread issues a tcgen05.mma about every 125 cycles whatever its width, and a 128 x 64 x 8 TF32 MMA runs in less:
+        // a plan may share a work item's columns between two issuing threads, each with accumulator columns and
+        // weight rows of its own.  With both operands in shared memory it does not pay (measured: 3-8 % slower on
+        // the layers of 128 channels per item, both threads read the same activation rows), so one thread is the default.
+        const int iss = warp >> 1;
+        if (lane == 0 && iss < cfg.n_iss) {
+            const int mma_n = cfg.bn / cfg.n_iss;
+            const uint32_t idesc = umma_idesc_tf32(BM, mma_n);
+            const uint32_t b_rows = static_cast<uint32_t>(iss * mma_n) * 128u;   // this issuer's weight rows inside a stage
             if (cfg.w_res && !mbar_wait(smem_u32(&s_wres), 0)) *abort_flag = 9;
             RingPos rp;
             uint32_t ab = 0, acc_par = 0;   // accumulator buffer of this item, parity of its current use
@@ -273,13 +281,13 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     break;
                 }
                 tc_fence_after();
-                const uint32_t acc = tmem + ab * cfg.bn;
+                const uint32_t acc = tmem + ab * cfg.bn + iss * mma_n;
                 for (int c = seg.sb; c < seg.se; ++c) {
                     if (!mbar_wait_lone(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     tc_fence_after();
                     const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
-                    uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * KBLK * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
+                    uint64_t bdesc = umma_desc_k_sw128((cfg.w_res ? wres + c * KBLK * cfg.b_bytes : a_smem + SUB_BYTES) + b_rows, 1024);
                     const uint32_t b_step = KBLK > 1 ? static_cast<uint32_t>(cfg.w_res ? cfg.b_bytes : cfg.sub_bytes) >> 4 : 0u;
 #pragma unroll
                     for (int j = 0; j < KBLK; ++j) {
@@ -570,6 +578,10 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     if (kblk > 2 || blk32 % kblk != 0) return false;
     cfg->kblk = kblk;
     cfg->n_sub = blk32 / kblk;
+    // one issuer thread unless the plan asks for two (halves of whole 8-row swizzle atoms, MMA widths multiples of 16)
+    const int n_iss = plan && plan->issuers > 0 ? plan->issuers : 1;
+    if (n_iss < 1 || n_iss > 2 || bn % (16 * n_iss) != 0) return false;
+    cfg->n_iss = n_iss;
     cfg->p_pad = static_cast<int>(((p.pixels + BM - 1) / BM) * BM);
     if (splits > 1 && (!p.splitk || p.splitk_bytes < static_cast<size_t>(splits) * cfg->p_pad * p.c_out * sizeof(float) ||
                        static_cast<long long>(splits) * cfg->p_pad >= (1ll << 31)))

@@ -36,6 +36,10 @@ def _plans(nm, s):
         p = nm.nm_plan_t()
         p.variant, p.bn, p.stages, p.split, p.kblk = 4, bn, stages, split, kblk
         out.append(p)
+    for bn, issuers in ((0, 1), (128, 1), (64, 2), (256, 2), (32, 2)):   # one and two MMA issuer threads
+        p = nm.nm_plan_t()
+        p.variant, p.bn, p.issuers = 4, bn, issuers
+        out.append(p)
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
     out.append(p)
