@@ -65,10 +65,12 @@ def source_digest(kernel: str) -> str:
         return hashlib.sha256(f.read()).hexdigest()[:16]
 
 
-def recorded_traffic(kernel: str, batch: int):
-    """DRAM bytes (read + write) of one step's launches of `kernel`, from the committed summary of an
-    ncu capture (profiles/dram_traffic_<kernel>.txt: key = value lines), scaled to `batch`; None if
-    there is no summary or the kernel source has changed since it was taken."""
+def recorded_traffic(kernel: str):
+    """DRAM bytes (read + write) per algorithmic byte of `kernel`, from the committed summary of single-layer ncu
+    captures (profiles/dram_traffic_<kernel>.txt: key = value lines); None if there is no summary or the kernel
+    source has changed since it was taken.  A launch's traffic is this ratio times its algorithmic bytes (the
+    captured layers' traffic grows with their bytes).  Output lines still dirty in the L2 when a kernel ends are
+    not in ncu's per-kernel write counter, so the figure bounds re-reads, not total writes."""
     path = os.path.join(ROOT, "profiles", f"dram_traffic_{kernel}.txt")
     if not os.path.exists(path):
         return None
@@ -81,7 +83,7 @@ def recorded_traffic(kernel: str, batch: int):
     try:
         if kv["source_sha256_16"] != source_digest(kernel):
             return None
-        return float(kv["dram_bytes_per_step"]) * batch / float(kv["batch"]), kv
+        return float(kv["dram_bytes_per_algorithmic_byte"])
     except (KeyError, ValueError):
         return None
 
@@ -622,11 +624,14 @@ def main():
         dom = max(by_kernel, key=lambda k: by_kernel[k]["ms"])
         d = by_kernel[dom]
         dom_gbs = d["bytes"] / (d["ms"] * 1e-3) / 1e9
-        traffic = recorded_traffic(dom, args.batch) if dom in KERNEL_SOURCE and not args.layer else None
+        traffic = recorded_traffic(dom) if dom in KERNEL_SOURCE else None
         out["roofline"] = {
             "bound": "hbm", "achieved": dom_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": dom_gbs / pk["hbm_gbs"],
-            # per launch, averaged over the launches of the profiled step (its plans may differ by a layer or two)
-            "traffic": traffic[0] / float(traffic[1].get("launches_per_step", d["launches"])) if traffic else None,
+            # per launch: DRAM bytes per algorithmic byte from single-layer ncu captures x this kernel's algorithmic bytes
+            # per launch (null once the kernel source has changed since the capture)
+            "traffic": traffic * d["bytes"] / d["launches"] if traffic else None,
+            "traffic_note": "scaled from single-layer captures (profiles/dram_traffic_<kernel>.txt); output lines still "
+                            "dirty in L2 at kernel end are not counted by the per-kernel write counter",
             "peak_source": pk["source"] + " (burst copy figure)",
             "kernel": dom, "launches_per_step": d["launches"], "avg_launch_ms": d["ms"] / d["launches"],
             "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],

@@ -71,11 +71,9 @@ def test_bench_host_logic(tmp_path, monkeypatch):
     assert len(bench.workload(8)) == 34 and bench.workload_name(8).startswith("mobilenet_v2_pointwise")
     monkeypatch.setitem(bench.WORKLOAD, "net", "resnet")
     # a traffic summary counts only while the kernel source it was taken from is unchanged
-    got = bench.recorded_traffic("k_conv_expand", 64)
+    got = bench.recorded_traffic("k_conv_expand")
     if got is not None:
-        total, kv = got
-        assert total == float(kv["dram_bytes_per_step"]) and kv["source_sha256_16"] == bench.source_digest("k_conv_expand")
-        assert bench.recorded_traffic("k_conv_expand", 128)[0] == 2 * total
+        assert 0.3 < got < 1.5          # DRAM bytes per algorithmic byte: no re-reads, some output still in L2
     monkeypatch.setattr(bench, "source_digest", lambda kernel: "0" * 16)
-    assert bench.recorded_traffic("k_conv_expand", 64) is None
-    assert bench.recorded_traffic("k_no_such_kernel", 64) is None
+    assert bench.recorded_traffic("k_conv_expand") is None
+    assert bench.recorded_traffic("k_no_such_kernel") is None
