@@ -657,12 +657,16 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     cfg->n_slices = p.n_tiles / g;
     cfg->n_acc = cfg->bn <= 128 ? 2 : 1;
     // MMA units: the item's accumulator columns cut into up to four pieces, none across two tiles
-    int sub = g == 1 ? 4 : g == 2 ? 2 : 1;
+    // (as many units as issuer threads asked for: a plan with fewer issuers gets wider MMAs)
+    const int want = plan && plan->issuers > 0 ? plan->issuers : MAX_ISS;
+    if (want > MAX_ISS) return false;
+    int sub = 1;
+    while (g * sub < want && sub < 4) sub *= 2;
     while (sub > 1 && (T % sub != 0 || (T / sub) % 16 != 0)) sub /= 2;
     cfg->mma_n = T / sub;
     cfg->n_units = g * sub;
-    int n_iss = plan && plan->issuers > 0 ? plan->issuers : (cfg->n_units < MAX_ISS ? cfg->n_units : MAX_ISS);
-    if (n_iss > cfg->n_units || n_iss > MAX_ISS) return false;
+    int n_iss = want < cfg->n_units ? want : cfg->n_units;
+    if (plan && plan->issuers > cfg->n_units) return false;
     cfg->n_iss = n_iss;
     cfg->kcp = KC <= 8 ? 8 : KC <= 16 ? 16 : 32;
     cfg->set_cols = g * cfg->kcp;
