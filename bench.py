@@ -39,10 +39,10 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 TF32_OVER_BF16 = 1.1 / 2.25   # nominal dense tensor peaks: 1.1 PFLOP/s TF32, 2.25 PFLOP/s bf16
 KERNEL_OF_VARIANT = {1: "k_conv_gather", 2: "k_conv_slab", 3: "k_conv_stream", 4: "k_conv_expand", 5: "k_conv_rowrun",
-                     6: "k_conv_window", 7: "k_conv_pair", 8: "k_conv_select"}
+                     6: "k_conv_window", 7: "k_conv_pair", 8: "k_conv_select", 9: "k_conv_planes"}
 KERNEL_SOURCE = {"k_conv_gather": "nm_conv_gather.cu", "k_conv_slab": "nm_conv_slab.cu", "k_conv_stream": "nm_conv_stream.cu",
                  "k_conv_expand": "nm_conv_expand.cu", "k_conv_rowrun": "nm_conv_rowrun.cu", "k_conv_window": "nm_conv_window.cu",
-                 "k_conv_pair": "nm_conv_pair.cu", "k_conv_select": "nm_conv_select.cu"}
+                 "k_conv_pair": "nm_conv_pair.cu", "k_conv_select": "nm_conv_select.cu", "k_conv_planes": "nm_conv_planes.cu"}
 KEPT_ONLY_VARIANTS = (1, 2, 3, 8)   # kernels that contract over the retained columns only (Algorithm 1 proper)
 PLAN_FIELDS = ("variant", "bn", "stages", "split", "kblk", "loads", "issuers", "ksplit")
 

@@ -90,6 +90,13 @@ typedef struct nm_weights nm_weights_t;
  *                whose output has the input's size, "patch" loads that fetch a pixel block and its halo
  *                once for all kh * kw taps.  `stages` = activation ring depth; `ksplit` > 1 splits the
  *                reduction axis like variant 4's split (same scratch, same second pass).
+ *            9 = plane kernel for at most four input channels and a horizontal stride of 1 or 2 (the 7x7 / 2
+ *                stem): the input rows of a band of output rows are held in shared memory with the channels
+ *                padded to four and, for stride 2, even and odd columns in separate planes, so that the tensor
+ *                core reads every tap's operand straight out of them (unswizzled K-major core matrices) and no
+ *                patch matrix is built (needs c_in <= 4, kw <= 8, dil_w = 1, stride_w 1 or 2, output rows of at
+ *                most 128 pixels, c_out % 32 == 0 and <= 256; any tile_t, any N:M).  `split` = output rows per
+ *                work item (1-4, 0 = as many as tensor memory holds), `stages` = row-band buffers (2 or 3).
  *   bn       output channels per CTA / work item (variants 2, 3, 8: a multiple of tile_t; variant 4: a
  *            multiple of 32 up to 256 that divides c_out rounded up to a multiple of 32; variant 6: a multiple
  *            of 32 up to 256 that divides c_out; variant 7: 128 or 256), 0 = default
@@ -102,7 +109,8 @@ typedef struct nm_weights nm_weights_t;
  *            one equal contiguous range per SM, an item shared by several CTAs is completed by the CTA
  *            that holds its first stage from the others' partial sums (per-SM slots in the same
  *            scratch; for layers with too few work items to fill every SM evenly);
- *            variant 6: M-tiles per work item (1-4); otherwise 0
+ *            variant 6: M-tiles per work item (1-4); variant 9: output rows per work item (1-4, 0 = most);
+ *            otherwise 0
  *   kblk     variants 4 and 7: 32-column blocks of the reduction axis per pipeline stage, 1 or 2 (0 = 1);
  *            two blocks halve the barrier round trips per MMA, which pays where the MMAs are short
  *            (few channels per work item) or the layer is small; K / 32 (per split) must be a multiple
@@ -115,7 +123,9 @@ typedef struct {
     int split;
     int kblk;
     int loads;    /* variant 8: 0 = the library's choice, 1 = im2col loads, 2 = patch loads */
-    int issuers;  /* MMA issuer threads: variant 8: 1-4 and at most the work item's MMA units (0 = as many as possible);
+    int issuers;  /* MMA issuer threads: variant 8: 1-4 (0 = 4); the work item's accumulator columns are cut into
+                     that many MMA units where the tile width allows (units of at least 16 columns, none across two
+                     tiles), so fewer issuers mean wider MMAs;
                      variant 4: 1 or 2, each with half of the item's channels (0 = 1) */
     int ksplit;   /* variant 8: ranges the reduction axis is split into, 1-8 (0 = 1); more than one needs scratch */
     int reserved[8];

@@ -38,6 +38,7 @@ void free_handle_memory(nm_weights* h)
     cudaFree(h->wx);
     cudaFree(h->w3);
     cudaFree(h->sel3);
+    cudaFree(h->ws);
     cudaFree(h->splitk);
     h->magic = 0;
     delete h;
@@ -133,6 +134,7 @@ nm_status_t make_params(const char* who, const nm_weights* w, const float* x, in
     p->w3 = w->w3;
     p->sel3 = w->sel3;
     p->sel_s = w->sel_s; p->sel_kc = w->sel_kc; p->sel_mw = w->sel_mw;
+    p->ws = w->ws;
     return NM_OK;
 }
 
@@ -161,6 +163,8 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
             return nmhost::launch_conv_pair(p, plan, st);
         case 8:
             return nmhost::launch_conv_select(p, plan, st);
+        case 9:
+            return nmhost::launch_conv_planes(p, plan, st);
         default:
             return nmhost::fail(NM_ERR_UNSUPPORTED, "nm_conv2d: unknown plan variant %d", variant);
     }
@@ -187,6 +191,11 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
             a.variant = 6; a.bn = bn; a.split = mt; a.stages = 0;
             if (nmhost::window_plan_ok(p, &a)) out.push_back(a);
         }
+    }
+    std::memset(&a, 0, sizeof(a));
+    for (int rows : {0, 2}) {               // plane kernel (at most four input channels, stride 1 or 2)
+        a.variant = 9; a.split = rows;
+        if (nmhost::planes_plan_ok(p, &a)) out.push_back(a);
     }
     std::memset(&a, 0, sizeof(a));
     a.variant = 5;                          // row-run kernel (few input channels)
@@ -303,6 +312,7 @@ nm_status_t nm_prune(const float* w_dense, int c_out, int kh, int kw, int c_in, 
     if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_expanded_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_select_layout(h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_planes_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         return s;
@@ -322,6 +332,7 @@ nm_status_t nm_weights_import(const float* values, const uint16_t* indices, int 
     if (s == NM_OK) s = nmhost::build_slab_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_expanded_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s == NM_OK) s = nmhost::build_select_layout(h, static_cast<cudaStream_t>(cuda_stream));
+    if (s == NM_OK) s = nmhost::build_planes_layout(h, static_cast<cudaStream_t>(cuda_stream));
     if (s != NM_OK) {
         free_handle_memory(h);
         *out = nullptr;

@@ -38,6 +38,8 @@ struct nm_weights {
     float* w3;           // [k / sel_s][c_out][32] TF32, rows swizzled (see k_build_w3)
     uint8_t* sel3;       // [k / sel_s][n_tiles][sel_mw bytes] select masks, 32-bit words (see k_build_sel3)
     int sel_s, sel_kc, sel_mw;
+    // Plane layout (variant 9): per kernel row a [c_out][32] tile of (kw, c) slots; NULL when the shape rules it out.
+    float* ws;           // [kh][c_out][32] TF32, rows swizzled (see k_build_ws)
 };
 
 // Geometry handed to the convolution kernels.
@@ -70,6 +72,8 @@ struct ConvParams {
     const float* w3;
     const uint8_t* sel3;
     int sel_s, sel_kc, sel_mw;
+    // plane layout (variant 9)
+    const float* ws;
 };
 
 #ifdef __CUDACC__
@@ -180,4 +184,9 @@ nm_status_t build_select_layout(nm_weights* h, cudaStream_t st);
 bool select_plan_ok(const ConvParams& p, const nm_plan_t* plan);
 size_t select_splitk_bytes(const ConvParams& p, int splits);
 nm_status_t launch_conv_select(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
+
+// nm_conv_planes.cu — variant 9
+nm_status_t build_planes_layout(nm_weights* h, cudaStream_t st);
+bool planes_plan_ok(const ConvParams& p, const nm_plan_t* plan);
+nm_status_t launch_conv_planes(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st);
 }  // namespace nmhost

@@ -43,6 +43,11 @@ def _plans(nm, s):
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
     out.append(p)
+    # plane kernel: as many output rows per item as fit, two rows with two band buffers, one row, three rows
+    for rows, stages in ((0, 0), (2, 2), (1, 0), (3, 3)):
+        p = nm.nm_plan_t()
+        p.variant, p.split, p.stages = 9, rows, stages
+        out.append(p)
     # window kernel: default, one M-tile with 64 channels, two / three / four M-tiles, short weight ring
     for bn, mt, stages in ((0, 0, 0), (64, 1, 0), (0, 2, 0), (32, 1, 3), (64, 3, 0), (32, 4, 0), (128, 4, 0)):
         p = nm.nm_plan_t()
@@ -160,6 +165,30 @@ def test_rowrun_shapes(nm, s):
 @pytest.mark.parametrize("s", ROWRUN[:4], ids=lambda s: s.name)
 def test_rowrun_shapes_integer_exact(nm, s):
     _run(nm, s, integer=True, need_variant=[5])
+
+
+# at most four input channels, horizontal stride 1 or 2, kernel rows of at most 8 taps: plane kernel
+PLANES = [
+    ConvShape("pl_stem", 2, 64, 64, 3, 64, 7, 7, 2, 3, 1, 1, 1, 64),
+    ConvShape("pl_stem_wide", 1, 40, 252, 3, 32, 7, 7, 2, 3, 1, 1, 1, 32),          # 126 output pixels per row
+    ConvShape("pl_ragged_band", 3, 30, 50, 3, 64, 7, 7, 2, 3, 1, 1, 1, 64),         # 15 output rows: a last band of three
+    ConvShape("pl_3x3_c4_s1", 2, 20, 20, 4, 64, 3, 3, 1, 1, 1, 2, 4, 8),             # stride 1, pruned, tile 8
+    ConvShape("pl_nopad_s1", 1, 24, 24, 4, 32, 3, 3, 1, 0, 1, 4, 4, 32),
+    ConvShape("pl_c1_5x5", 2, 31, 31, 1, 32, 5, 5, 2, 2, 1, 1, 1, 32),               # one channel, odd sizes
+    ConvShape("pl_c2_3x8", 1, 18, 40, 2, 128, 3, 8, 2, 3, 1, 1, 1, 32),              # eight taps per kernel row, two rows per item
+    ConvShape("pl_c256", 1, 16, 16, 3, 256, 3, 3, 1, 1, 1, 1, 1, 64),                # 256 channels: one output row per item
+    ConvShape("pl_stem_224", 1, 224, 224, 3, 64, 7, 7, 2, 3, 1, 1, 1, 64),           # the ResNet stem at full size
+]
+
+
+@pytest.mark.parametrize("s", PLANES, ids=lambda s: s.name)
+def test_plane_shapes(nm, s):
+    _run(nm, s, need_variant=[9])
+
+
+@pytest.mark.parametrize("s", PLANES[:8], ids=lambda s: s.name)
+def test_plane_shapes_integer_exact(nm, s):
+    _run(nm, s, integer=True, need_variant=[9])
 
 
 # stride-1 spatial kernels with c_in and c_out multiples of 32: window kernel
