@@ -144,6 +144,7 @@ nm_status_t run_plan(const ConvParams& p, const nm_plan_t* plan, cudaStream_t st
     switch (variant) {
         case 0:
             if (nmhost::stream_plan_ok(p, nullptr)) return nmhost::launch_conv_stream(p, nullptr, st);
+            if (nmhost::planes_plan_ok(p, nullptr)) return nmhost::launch_conv_planes(p, nullptr, st);
             if (p.c_in % 32 != 0 && nmhost::rowrun_plan_ok(p, nullptr)) return nmhost::launch_conv_rowrun(p, nullptr, st);
             if (nmhost::slab_plan_ok(p, nullptr)) return nmhost::launch_conv_slab(p, nullptr, st);
             return nmhost::launch_conv_gather(p, st);

@@ -19,8 +19,11 @@
 //                            MMAs against the weights, which stay in shared memory for the whole kernel
 //                            (per kernel row a [C_out x 32] swizzled tile: kw padded to 8 taps, channels to 4,
 //                            zeros in the padding and in pruned columns, so any N:M and tile width works)
-//   epilogue (8 warps)       TMEM -> registers, + bias (+ shortcut), ReLU, staged and stored with TMA; pixels
-//                            past the end of the output row are clipped by the store's bounds check
+//   epilogue (16 warps)      four per output row of the band (one per 32 accumulator lanes): TMEM -> registers,
+//                            + bias (+ shortcut), ReLU, staged and stored with TMA; pixels past the end of the
+//                            output row are clipped by the store's bounds check.  A 32 x 32 block takes a warp
+//                            about 2 k cycles of latencies in series (TMEM load, staging, proxy fence, store),
+//                            hence a warp per (row, lane quarter): the epilogue of an item is two blocks deep
 // A work item is (image, band of R output rows); persistent CTAs, static schedule; accumulators and planes
 // are double-buffered; every wait is bounded and reports through the handle's status word.
 #include "nm_internal.h"
@@ -34,10 +37,10 @@ using namespace nmk;
 constexpr int BM = 128;
 constexpr int MAX_R = 4;            // output rows per work item = MMA issuer threads
 constexpr int LOAD_WARPS = 8;
-constexpr int EPI_WARPS = 8;
-constexpr int THREADS = (4 + EPI_WARPS + LOAD_WARPS) * 32;   // warps 0-3 issuers, 4-11 epilogue, 12-19 loaders
+constexpr int EPI_WARPS = 4 * MAX_R;
+constexpr int THREADS = (4 + EPI_WARPS + LOAD_WARPS) * 32;   // warps 0-3 issuers, 4-19 epilogue, 20-27 loaders
 constexpr int MAX_SLOTS = 3;
-constexpr int STAGING_BYTES = EPI_WARPS * 2 * 4096;
+constexpr int STAGING_BYTES = EPI_WARPS * 4096;             // one 32 x 32 box per epilogue warp
 constexpr int LOAD_UNROLL = 6;
 
 struct PlaneCfg {
@@ -55,18 +58,6 @@ struct PlaneCfg {
 };
 
 __device__ __forceinline__ bool aborted(volatile int* flag) { return *flag != 0; }
-
-// Shared-memory operand descriptor, K-major, no swizzle: core matrices of 8 rows x 16 bytes (128 contiguous
-// bytes), `lbo_bytes` between the two core matrices along K, `sbo_bytes` between 8-row groups.
-__device__ __forceinline__ uint64_t umma_desc_k_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
-    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= static_cast<uint64_t>(1) << 46;   // descriptor version for sm_100; layout field 0 = no swizzle
-    return d;
-}
 
 template <int S>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -147,12 +138,16 @@ k_conv_planes(const ConvParams p, const PlaneCfg cfg, const __grid_constant__ CU
         }
     } else if (warp < 4 + EPI_WARPS) {
         // =========================== epilogue ===========================
-        const int q = warp & 3, grp = (warp - 4) >> 2;
+        const int q = warp & 3, mi = (warp - 4) >> 2;   // TMEM lane quarter, output row of the band
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const uint32_t my_staging = staging + (warp - 4) * 2 * 4096;
+        const uint32_t box = staging + (warp - 4) * 4096;
+        const uint32_t stage_row = box + lane * 128;
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = p.c_out / 32;
+        const bool has_row = mi < cfg.r;
         uint32_t nb = 0, ti = 0;
+        // the bias of a block is held one value per lane and fetched a block ahead (it is the same for every item)
+        float bias_next = has_row ? bias_lane_load(p.bias, 0, p.c_out, lane) : 0.f;
         for (uint32_t work = blockIdx.x; work < n_work; work += gridDim.x, ++ti) {
             const int ab = static_cast<int>(ti & 1u);
             const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
@@ -160,55 +155,54 @@ k_conv_planes(const ConvParams p, const PlaneCfg cfg, const __grid_constant__ CU
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
             const int n = static_cast<int>(work / static_cast<uint32_t>(cfg.bands));
-            const int oh0 = static_cast<int>(work - static_cast<uint32_t>(n) * static_cast<uint32_t>(cfg.bands)) * cfg.r;
-            bool released = false;
-            for (int mi = grp; mi < cfg.r; mi += 2) {
-                const int oh = oh0 + mi;
-                const bool row_ok = oh < p.ho;
-                const long long row_pixel0 = (static_cast<long long>(n) * p.ho + oh) * p.wo;
-                for (int blk = 0; blk < n_blk; ++blk, ++nb) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + ab * cfg.acc_cols + mi * p.c_out + blk * 32, v);
-                    tmem_ld_wait();
-                    if (mi + 2 >= cfg.r && blk == n_blk - 1) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
-                        released = true;
-                    }
-                    const uint32_t box = my_staging + (nb & 1u) * 4096;
-                    if (lane == 0 && nb >= 2) tma_store_wait_read_n<1>();
+            const int oh = static_cast<int>(work - static_cast<uint32_t>(n) * static_cast<uint32_t>(cfg.bands)) * cfg.r + mi;
+            const bool row_ok = has_row && oh < p.ho;
+            const bool box_ok = row_ok && q * 32 < p.wo;
+            const long long box_pixel = (static_cast<long long>(n) * p.ho + oh) * p.wo + q * 32;
+            const int box_rows = p.wo - q * 32 < 32 ? p.wo - q * 32 : 32;
+            for (int blk = 0; has_row && blk < n_blk; ++blk, ++nb) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_addr + ab * cfg.acc_cols + mi * p.c_out + blk * 32, v);
+                const float bias_cur = bias_next;
+                bias_next = bias_lane_load(p.bias, blk + 1 < n_blk ? (blk + 1) * 32 : 0, p.c_out, lane);
+                if (lane == 0 && nb >= 1) tma_store_wait_read();   // the store that last read the box is done with it
+                __syncwarp();
+                tmem_ld_wait();
+                if (blk == n_blk - 1) {
+                    tc_fence_before();
                     __syncwarp();
-                    const uint32_t stage_row = box + lane * 128;
-                    const float4* rrow = nm_residual_row(p, row_ok && q * 32 + lane < p.wo ? row_pixel0 + q * 32 + lane : p.pixels, blk * 32);
+                    if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+                }
+                const int relu_now = p.residual ? 0 : p.relu;   // with a shortcut input the activation follows the addition
 #pragma unroll
-                    for (int qq = 0; qq < 8; ++qq) {
-                        float o[4];
-                        float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + blk * 32) + qq);
-                        if (rrow) nm_add4(bv, __ldg(rrow + qq));
-                        o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
-                        o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
-                        o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
-                        o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
-                        if (p.relu) {
+                for (int qq = 0; qq < 8; ++qq) {
+                    float o[4];
+                    const float4 bv = bias_quad(bias_cur, qq);
+                    o[0] = __uint_as_float(v[qq * 4 + 0]) + bv.x;
+                    o[1] = __uint_as_float(v[qq * 4 + 1]) + bv.y;
+                    o[2] = __uint_as_float(v[qq * 4 + 2]) + bv.z;
+                    o[3] = __uint_as_float(v[qq * 4 + 3]) + bv.w;
+                    if (relu_now) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
-                        }
-                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage_row + ((qq ^ rx) << 4)), "f"(o[0]),
-                                     "f"(o[1]), "f"(o[2]), "f"(o[3])
-                                     : "memory");
+                        for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
                     }
-                    fence_proxy_async();
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage_row + ((qq ^ rx) << 4)), "f"(o[0]),
+                                 "f"(o[1]), "f"(o[2]), "f"(o[3])
+                                 : "memory");
+                }
+                if (p.residual && box_ok) {
                     __syncwarp();
-                    if (lane == 0) {
-                        // output seen as (channel, ow, n * ho + oh): pixels past the row's end are clipped
-                        if (row_ok && q * 32 < p.wo) tma_store_3d(&tm_y, box, blk * 32, q * 32, n * p.ho + oh);
-                        tma_store_commit();
-                    }
+                    add_residual_box(box, p.residual + box_pixel * p.c_out + blk * 32, p.c_out, box_rows, p.relu, lane);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    // output seen as (channel, ow, n * ho + oh): pixels past the row's end are clipped
+                    if (box_ok) tma_store_3d(&tm_y, box, blk * 32, q * 32, n * p.ho + oh);
+                    tma_store_commit();
                 }
             }
-            if (!released) {   // a band of one row: the second group has nothing to read
+            if (!has_row) {   // a band of fewer rows than warps: nothing to read
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));

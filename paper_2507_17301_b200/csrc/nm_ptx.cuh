@@ -361,6 +361,18 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t addr, uint32_t sb
     d |= static_cast<uint64_t>(2) << 61;                          // layout: 128-byte swizzle
     return d;
 }
+// Shared-memory operand descriptor, K-major, no swizzle: core matrices of 8 rows x 16 bytes (128 contiguous
+// bytes), `lbo_bytes` between the two core matrices along K, `sbo_bytes` between 8-row groups.
+__device__ __forceinline__ uint64_t umma_desc_k_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;   // descriptor version for sm_100; layout field 0 = no swizzle
+    return d;
+}
+
 // Instruction descriptor: TF32 x TF32 -> fp32, both operands K-major, shape m x n (x 8).
 __host__ __device__ constexpr uint32_t umma_idesc_tf32(int m, int n)
 {

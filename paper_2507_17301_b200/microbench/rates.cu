@@ -125,11 +125,21 @@ __global__ void __launch_bounds__(256, 1) k_mma(int count, int n, int issuers, i
     const long long t0 = clock64();
     if (warp < issuers && lane == 0) {
         const uint32_t idesc = umma_idesc_tf32(128, n);
-        const uint64_t bdesc = umma_desc_k_sw128(base, 1024), adesc = umma_desc_k_sw128(base + 32768, 1024);
+        // operand layouts: 128-byte-swizzled K-major rows, or unswizzled K-major core matrices (8 rows x 16 bytes = 128
+        // contiguous bytes; 128 bytes between 8-row groups; A: 1856 bytes between the two core matrices along K, as in the
+        // plane kernel; B: n * 16 bytes, i.e. a [K / 4][n][16 bytes] image)
+        const uint64_t a_sw = umma_desc_k_sw128(base + 32768, 1024), a_pl = umma_desc_k_plain(base + 32768, 1856, 128);
+        const uint64_t b_sw = umma_desc_k_sw128(base, 1024), b_pl = umma_desc_k_plain(base, n * 16, 128);
+        const uint32_t b_step = static_cast<uint32_t>(2 * n);   // two core-matrix columns of B, in 16-byte units
         const uint32_t acc = tmem + warp * (256 / issuers);   // 256 / issuers >= n
+        // B unswizzled inside the 1 KB atoms of the swizzled layout ([8 rows][128 bytes] stored as [8 K pieces][8 rows][16 bytes]):
+        // 128 bytes between core matrices along K, 1024 between 8-row groups; a run of rows stays one contiguous copy
+        const uint64_t b_at = umma_desc_k_plain(base, 128, 1024);
+        const bool a_plain = (ss & 2) != 0, b_plain = (ss & 4) != 0, b_atom = (ss & 8) != 0;
         for (int i = 0; i < count; ++i) {
-            if (ss) umma_tf32_ss(acc, adesc + 2 * (i & 3), bdesc + 2 * (i & 3), idesc, 1u);
-            else umma_tf32_ts(acc, tmem + 256 + (i & 7) * 8, bdesc + 2 * (i & 3), idesc, 1u);
+            const uint64_t bd = b_atom ? b_at + 16 * (i & 3) : b_plain ? b_pl + (i & 3) * b_step : b_sw + 2 * (i & 3);
+            if (ss & 1) umma_tf32_ss(acc, a_plain ? a_pl + (i & 3) : a_sw + 2 * (i & 3), bd, idesc, 1u);
+            else umma_tf32_ts(acc, tmem + 256 + (i & 7) * 8, bd, idesc, 1u);
         }
         umma_commit(smem_u32(&s_done[warp]));
         if (!mbar_wait(smem_u32(&s_done[warp]), 0)) std::printf("wait expired\n");
@@ -192,7 +202,9 @@ int main()
             }
         }
     }
-    for (int ss : {0, 1}) {
+    const char* names[12] = {"TS", "SS", "", "SS plain A", "TS plain B", "SS plain B", "", "SS plain A, B",
+                             "TS atom B", "SS atom B", "", "SS plain A, atom B"};
+    for (int ss : {0, 4, 8, 1, 3, 5, 7, 9, 11}) {   // bit 0: A from shared memory, bit 1: A unswizzled, bit 2: B unswizzled
         for (int n : {64, 128, 256}) {
             for (int issuers : {1, 2, 4}) {
                 if (256 / issuers < n) continue;
@@ -200,7 +212,7 @@ int main()
                 const float ms = best_ms([&] { k_mma<<<sms, 256, smem>>>(count, n, issuers, ss, cyc); });
                 CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
                 const double total = static_cast<double>(count) * issuers;
-                std::printf("mma     %s N=%3d issuers=%d : %6.1f cycles per MMA, %6.1f ns, %5.0f TFLOP/s over %d SMs\n", ss ? "SS" : "TS", n,
+                std::printf("mma     %s N=%3d issuers=%d : %6.1f cycles per MMA, %6.1f ns, %5.0f TFLOP/s over %d SMs\n", names[ss], n,
                             issuers, static_cast<double>(h) / total, ms * 1e6 / total,
                             sms * total * 128.0 * n * 8 * 2 / (ms * 1e-3) / 1e12, sms);
             }
