@@ -565,7 +565,7 @@ def main():
             t_roof_sum += t_roof
             table.append({"layer": s.name, "shape": f"{s.c_in}->{s.c_out} {s.kh}x{s.kw}/{s.stride} @{s.h}",
                           "ms": round(ms, 4), "ms_warm": round(warm_ms, 4) if warm_ms is not None else None,
-                          "kept_columns_only": plan.variant in KEPT_ONLY_VARIANTS,
+                          "kept_columns_only": plan.variant in KEPT_ONLY_VARIANTS or s.n_keep == s.m_group,
                           "useful_tflops": round(useful_flops(s) / (ms * 1e-3) / 1e12, 2),
                           "gbs": round(algorithmic_bytes(s) / (ms * 1e-3) / 1e9, 1),
                           "bound": "tensor" if t_tc > t_hbm else "hbm", "roofline_frac": round(t_roof / ms, 3),
@@ -650,6 +650,9 @@ def main():
             os.environ["NM_AUTOTUNE_VARIANTS"] = ",".join(str(v) for v in KEPT_ONLY_VARIANTS)
             gplans = []
             for s, hnd, x, bias, y, plan in state:
+                if s.n_keep == s.m_group:     # an unpruned layer (the stem) has no pruned columns to skip: any kernel qualifies
+                    gplans.append(plan)
+                    continue
                 gp, _ = nm.nm_autotune(hnd, x, s.stride, s.pad, s.dil, bias, s.relu, y_scratch=y, kh=s.kh, kw=s.kw)
                 gplans.append(gp)
             del os.environ["NM_AUTOTUNE_VARIANTS"]
@@ -669,9 +672,10 @@ def main():
             g_ms = a.elapsed_time(b) / args.steps
             out["gather_only"] = {"value": args.batch / (g_ms * 1e-3), "unit": UNIT, "ms_per_step": g_ms,
                                   "useful_tflops": flops_step / (g_ms * 1e-3) / 1e12,
-                                  "variants": {str(v): sum(1 for gp in gplans if gp.variant == v) for v in KEPT_ONLY_VARIANTS},
+                                  "variants": {str(v): sum(1 for gp in gplans if gp.variant == v) for v in sorted({gp.variant for gp in gplans})},
                                   "note": "plans restricted to the kernels that contract over the retained columns only "
-                                          "(variants 1-3 and 8: Algorithm 1 proper); the headline lets the tuner also take the "
+                                          "(variants 1-3 and 8: Algorithm 1 proper); unpruned layers (the stem) keep their plan, "
+                                          "they have no pruned column; the headline lets the tuner also take the "
                                           "expanded-operand kernels, which multiply the zeros of the pruned columns"}
 
         # the same layers chained as the network's dataflow: stem -> max-pool -> residual blocks, every
