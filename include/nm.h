@@ -109,7 +109,8 @@ typedef struct nm_weights nm_weights_t;
  *            one equal contiguous range per SM, an item shared by several CTAs is completed by the CTA
  *            that holds its first stage from the others' partial sums (per-SM slots in the same
  *            scratch; for layers with too few work items to fill every SM evenly);
- *            variant 6: M-tiles per work item (1-4); variant 9: output rows per work item (1-4, 0 = most);
+ *            variant 6: M-tiles per work item (1-4); variant 8: 1 = four epilogue warps, 2 = eight (0 = eight where a
+ *            work item has at most four chunks); variant 9: output rows per work item (1-4, 0 = most);
  *            otherwise 0
  *   kblk     variants 4 and 7: 32-column blocks of the reduction axis per pipeline stage, 1 or 2 (0 = 1);
  *            two blocks halve the barrier round trips per MMA, which pays where the MMAs are short

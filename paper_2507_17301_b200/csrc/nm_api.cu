@@ -182,8 +182,10 @@ std::vector<nm_plan_t> candidate_plans(const nm_weights* /*w*/, const ConvParams
     // items exist (the split plans need the handle's scratch)
     for (int ksplit : {1, 2, 3, 4}) {
         for (int bn : {256, 128, 64}) {
-            a.variant = 8; a.bn = bn; a.ksplit = ksplit;
-            if (bn % p.tile_t == 0 && nmhost::select_plan_ok(p, &a)) out.push_back(a);
+            for (int epi : {1, 2}) {        // four or eight epilogue warps (split plans: the library's choice)
+                a.variant = 8; a.bn = bn; a.ksplit = ksplit; a.split = ksplit == 1 ? epi : 0;
+                if ((ksplit == 1 || epi == 1) && bn % p.tile_t == 0 && nmhost::select_plan_ok(p, &a)) out.push_back(a);
+            }
         }
     }
     std::memset(&a, 0, sizeof(a));

@@ -33,7 +33,7 @@
 //                         are T TMEM columns).  A lone thread issues an MMA every ~125 cycles whatever its
 //                         size, a 128 x 64 x 8 MMA runs in 35: the units of an item are dealt to up to four
 //                         issuer threads, each with accumulator columns of its own.
-//   epilogue (4 warps)    TMEM -> registers, + bias, (+ shortcut), ReLU, staged through shared memory
+//   epilogue (8 warps)    TMEM -> registers, + bias, (+ shortcut), ReLU, staged through shared memory
 //                         and written to NHWC with TMA stores; with two accumulator buffers it
 //                         overlaps the next item's main loop.
 //
@@ -49,13 +49,14 @@ using namespace nmk;
 
 constexpr int BM = 128;
 constexpr int THREADS = 576;   // warps: 0 activation producer, 1 weight producer, 2 3 16 17 MMA issuers, 4-7 epilogue, 8-15 compactors
+constexpr int THREADS_EPI8 = 704;   // ... and four more epilogue warps, 18-21 (the registers per thread then drop from 96 to 80)
 constexpr int MAX_P = 4;       // activation ring slots
 constexpr int MAX_W = 8;       // weight ring slots
 constexpr int MAX_SETS = 4;    // operand sets in tensor memory
 constexpr int MAX_ISS = 4;
 constexpr int MAX_TAPS = 32;
 constexpr int A_COL0 = 256;    // TMEM: accumulators in columns [0, 256), operand sets above
-constexpr int STAGING_BYTES = 4 * 2 * 4096;
+constexpr int STAGING_BYTES = 4 * 2 * 4096;   // two boxes per epilogue warp (twice that with eight epilogue warps)
 
 struct SelCfg {
     int g, bn, n_slices, n_acc, n_iss;
@@ -72,6 +73,7 @@ struct SelCfg {
     int wstage_bytes;   // w_bytes + m_bytes rounded up to 1024
     int n_p, n_w, n_sets, kcp, set_cols;
     int ksplit, p_pad;
+    int epi8;           // eight epilogue warps instead of four
     int alias_staging;  // 1: the output staging boxes lie over the start of the activation ring (one work item per CTA)
     int boxes;          // staging boxes (32 pixels x 32 channels) per epilogue warp: 2, or one per channel block when aliased
     int n_act;          // activation stages per work item
@@ -151,8 +153,8 @@ __device__ __forceinline__ Item item_of(uint32_t work, const SelCfg& cfg)
     return it;
 }
 
-template <int NK, int MG>
-__global__ void __launch_bounds__(THREADS, 1)
+template <int NK, int MG, int EPI8>
+__global__ void __launch_bounds__(EPI8 ? THREADS_EPI8 : THREADS, 1)
 k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUtensorMap tm_x,
               const __grid_constant__ CUtensorMap tm_y)
 {
@@ -195,7 +197,7 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&s_accfull[i]), cfg.n_iss);
-            mbar_init(smem_u32(&s_accfree[i]), 4);            // epilogue warps
+            mbar_init(smem_u32(&s_accfree[i]), EPI8 ? 8 : 4);  // epilogue warps
         }
         mbar_fence_init();
         s_abort = 0;
@@ -354,11 +356,17 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp >= 4 && warp < 8) {
+    } else if ((warp >= 4 && warp < 8) || (EPI8 && warp >= 18)) {
         // =========================== epilogue ===========================
+        // With eight epilogue warps two warps per 32 accumulator lanes take alternate 32-channel blocks: a block costs
+        // a warp about a thousand cycles of latencies in series (TMEM load, staging, proxy fence, store), so the warps,
+        // not their instructions, set the pace of an item's epilogue.  It pays where an item has few chunks (pointwise
+        // layers with many output channels); elsewhere the compactors need the registers the extra warps take.
         const int q = warp & 3;
+        constexpr int ESTEP = EPI8 ? 2 : 1;
+        const int half = warp >= 18 ? 1 : 0;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const uint32_t my_staging = staging + q * cfg.boxes * 4096;
+        const uint32_t my_staging = staging + (half * 4 + q) * cfg.boxes * 4096;
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t ti = 0;
@@ -377,19 +385,24 @@ k_conv_select(const ConvParams p, const SelCfg cfg, const __grid_constant__ CUte
             const long long box_pix = static_cast<long long>(it.pix0) + q * 32;
             const int store_row = it.split * cfg.p_pad + static_cast<int>(it.pix0) + q * 32;
             const bool in_range = cfg.ksplit > 1 || box_pix < p.pixels;
-            for (int blk = 0; blk < n_blk; ++blk, ++nb) {
+            if (EPI8 && half >= n_blk) {   // a single channel block: the second warp of the quarter only releases the buffer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
+            }
+            for (int blk = half; blk < n_blk; blk += ESTEP, ++nb) {
                 const float bias_l = bias_lane_load(p.bias, o0 + blk * 32, p.c_out, lane);
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_addr + ab * cfg.bn + blk * 32, v);
                 tmem_ld_wait();
-                if (blk == n_blk - 1) {
+                if (blk + ESTEP >= n_blk) {
                     // the accumulator buffer may be overwritten from here on
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&s_accfree[ab]));
                 }
                 // two boxes: the box's previous store (two blocks ago) has read it; a box per block: nothing to wait for
-                const uint32_t box = my_staging + (cfg.boxes == 2 ? (nb & 1u) : static_cast<uint32_t>(blk)) * 4096;
+                const uint32_t box = my_staging + (cfg.boxes == 2 ? (nb & 1u) : static_cast<uint32_t>(blk / ESTEP)) * 4096;
                 if (cfg.boxes == 2 && lane == 0 && nb >= 2) tma_store_wait_read_n<1>();
                 __syncwarp();
                 const uint32_t stage_row = box + lane * 128;
@@ -694,8 +707,12 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     cfg->n_work = pix_blocks * cfg->n_slices * ksplit;
     if (cfg->n_work >= (1ll << 31)) return false;
     cfg->alias_staging = cfg->n_work <= sm_count();
+    // epilogue warps: plan.split = 1 four, 2 eight, 0 eight where an item has few chunks and several channel blocks
+    if (plan && (plan->split < 0 || plan->split > 2)) return false;
+    cfg->epi8 = plan && plan->split > 0 ? plan->split == 2 : (cfg->n_act * cfg->taps <= 4 && cfg->bn >= 64);
+    const int staging_bytes = cfg->epi8 ? 2 * STAGING_BYTES : STAGING_BYTES;
     // alignment slack, static shared, and the output staging unless it can lie over the ring
-    const int budget = 227 * 1024 - 1024 - 4096 - (cfg->alias_staging ? 0 : STAGING_BYTES);   // static: barriers, 1 KB of zero rows and their alignment
+    const int budget = 227 * 1024 - 1024 - 4096 - (cfg->alias_staging ? 0 : staging_bytes);   // static: barriers, 1 KB of zero rows and their alignment
     const bool paired = cfg->taps == 1;
     int n_p = 2;
     if (plan && plan->stages > 0) n_p = plan->stages;
@@ -716,8 +733,9 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, SelCfg* cfg)
     if (cfg->alias_staging) {
         // one work item per CTA: the rings are idle when the epilogue runs, every channel block gets a box of its own
         const int ring_bytes = n_p * cfg->p_bytes + n_w * cfg->wstage_bytes;
-        if (ring_bytes >= 4 * (cfg->bn / 32) * 4096) cfg->boxes = cfg->bn / 32;
-        else if (ring_bytes < STAGING_BYTES) cfg->alias_staging = 0;
+        const int warps = cfg->epi8 ? 8 : 4, per_warp = (cfg->bn / 32 + (cfg->epi8 ? 1 : 0)) / (cfg->epi8 ? 2 : 1);
+        if (per_warp >= 2 && ring_bytes >= warps * per_warp * 4096) cfg->boxes = per_warp;   // a box per block the warp handles
+        else if (ring_bytes < staging_bytes) cfg->alias_staging = 0;
     }
     return true;
 }
@@ -751,12 +769,13 @@ nm_status_t launch(const ConvParams& p, const SelCfg& cfg, cudaStream_t st)
         return nmhost::fail(NM_ERR_CUDA, "nm_conv2d: tensor-map encoding failed (variant 8)");
     q.pixels = p.pixels;
     size_t smem = 1024 + static_cast<size_t>(cfg.n_p) * cfg.p_bytes + static_cast<size_t>(cfg.n_w) * cfg.wstage_bytes +
-                  (cfg.alias_staging ? 0 : STAGING_BYTES);
+                  (cfg.alias_staging ? 0 : (cfg.epi8 ? 2 : 1) * STAGING_BYTES);
     if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: it owns all 512 TMEM columns
-    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(k_conv_select<NK, MG>), smem);
+    const auto kernel = cfg.epi8 ? k_conv_select<NK, MG, 1> : k_conv_select<NK, MG, 0>;
+    cudaError_t e = nmhost::ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "cudaFuncSetAttribute (variant 8): %s", cudaGetErrorString(e));
     const long long grid = cfg.n_work < sm_count() ? cfg.n_work : sm_count();
-    e = nmhost::launch_pdl(k_conv_select<NK, MG>, static_cast<unsigned>(grid), THREADS, smem, st, q, cfg, tm_x, tm_y);
+    e = nmhost::launch_pdl(kernel, static_cast<unsigned>(grid), cfg.epi8 ? THREADS_EPI8 : THREADS, smem, st, q, cfg, tm_x, tm_y);
     nmhost::count_launch(1);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return nmhost::fail(NM_ERR_CUDA, "nm_conv2d launch (variant 8): %s", cudaGetErrorString(e));

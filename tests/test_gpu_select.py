@@ -30,7 +30,9 @@ def _plans(nm, s):
     t = s.tile_t
     return [_plan(nm), _plan(nm, loads=1), _plan(nm, loads=2), _plan(nm, bn=t), _plan(nm, bn=t, loads=1, stages=2),
             _plan(nm, bn=2 * t, issuers=1), _plan(nm, bn=4 * t, issuers=2, loads=1), _plan(nm, bn=4 * t, loads=2, stages=1), _plan(nm, loads=1, stages=4),
-            _plan(nm, bn=256), _plan(nm, bn=128, loads=2)]
+            _plan(nm, bn=256), _plan(nm, bn=128, loads=2),
+            # four and eight epilogue warps (split = 1, 2; the default picks by the item's chunk count)
+            _plan(nm, split=1), _plan(nm, split=2), _plan(nm, bn=t, split=2, loads=1), _plan(nm, bn=256, split=2), _plan(nm, bn=2 * t, split=1, issuers=2)]
 
 
 # name, batch, h, w, c_in, c_out, kh, kw, stride, pad, dil, N, M, T
@@ -134,7 +136,7 @@ def test_select_kernel_with_shortcut(nm):
     yr = oracle.conv2d_res(vr, ir, 3, 3, s.c_in, 64, x.numpy(), (1, 1), (1, 1), (1, 1), b.numpy(), res.numpy(), True)
     hnd = nm.nm_prune(w.cuda(), 2, 4, 64)
     nm.nm_weights_reserve(hnd, 2 * 640 * 128 * 4)
-    for plan in (_plan(nm), _plan(nm, loads=1, bn=64), _plan(nm, ksplit=2)):
+    for plan in (_plan(nm), _plan(nm, loads=1, bn=64), _plan(nm, ksplit=2), _plan(nm, split=1), _plan(nm, split=2)):
         y = nm.nm_conv2d(hnd, x.cuda(), 3, 3, 1, 1, 1, b.cuda(), True, plan=plan, residual=res.cuda())
         nm.nm_weights_check(hnd)
         torch.cuda.synchronize()
