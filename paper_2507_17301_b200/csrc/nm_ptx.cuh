@@ -373,6 +373,13 @@ __device__ __forceinline__ uint64_t umma_desc_k_plain(uint32_t addr, uint32_t lb
     return d;
 }
 
+// Copies 128 rows x 256 bits (8 fp32 per row) of a shared-memory operand tile, described like an MMA operand, into 8
+// tensor-memory columns (row r -> lane r).  Issued by one thread; runs in order with that thread's MMAs and is
+// covered by its next tcgen05.commit.
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t sdesc)
+{
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
 // Instruction descriptor: TF32 x TF32 -> fp32, both operands K-major, shape m x n (x 8).
 __host__ __device__ constexpr uint32_t umma_idesc_tf32(int m, int n)
 {

@@ -6,6 +6,8 @@
 //            loaded from shared memory), byte masks (one byte per select, widened with a byte permute).
 //   mma      TF32 tcgen05.mma of shape 128 x N x 8 issued back to back by 1, 2 or 4 threads (each with accumulator
 //            columns of its own), A from tensor memory (TS) or from shared memory (SS).
+//   cp       tcgen05.cp of an operand tile from shared to tensor memory: layout check, issue rate, and the rate of
+//            the pattern "four copies, four TS MMAs" per 32-column block from one and from two threads.
 //
 // Prints cycles per unit of work from clock64 and from CUDA events.  Nothing here is used by the library.
 #include <cstdio>
@@ -151,6 +153,98 @@ __global__ void __launch_bounds__(256, 1) k_mma(int count, int n, int issuers, i
     if (warp == 7) tmem_dealloc(tmem, 512);
 }
 
+
+// MODE 0: layout check (a swizzled 128 x 32 tile with element (row, col) = row * 32 + col is copied with four
+// tcgen05.cp and read back; prints the number of mismatches).  MODE 1: `count` copies back to back from one thread.
+// MODE 2: per 32-column block four copies then four 128 x n x 8 TS MMAs on the copied columns, one thread.
+// MODE 3: the same with the copies issued by a second thread (hand-over through mbarriers, four operand slots).
+__global__ void __launch_bounds__(256, 1) k_cp(int mode, int count, int n, long long* cycles, int* mismatches)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem;
+    __shared__ uint64_t s_done[2], s_ready[4], s_free[4];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // B region (32 KB of zeros) at base, A tile at base + 32768: row r = 128 bytes, 16-byte pieces XOR-ed with r % 8
+    for (int i = tid; i < 8192; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw + (base - smem_u32(smem_raw)))[i] = 0;
+    for (int i = tid; i < 128 * 32; i += blockDim.x) {
+        const int r = i >> 5, c = i & 31;
+        const uint32_t off = 32768u + r * 128u + ((static_cast<uint32_t>(c >> 2) ^ static_cast<uint32_t>(r & 7)) << 4) + (c & 3) * 4u;
+        *reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)) + off) = static_cast<float>(i);
+    }
+    if (warp == 7) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) mbar_init(smem_u32(&s_done[i]), 1);
+        for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&s_ready[i]), 1); mbar_init(smem_u32(&s_free[i]), 1); }
+        mbar_fence_init();
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const uint64_t a_sw = umma_desc_k_sw128(base + 32768, 1024), b_sw = umma_desc_k_sw128(base, 1024);
+    const uint32_t idesc = umma_idesc_tf32(128, n);
+    const long long t0 = clock64();
+    if (mode == 0) {
+        if (tid == 0) {
+            for (int kq = 0; kq < 4; ++kq) tmem_cp_128x256b(tmem + 256 + kq * 8, a_sw + 2 * kq);
+            umma_commit(smem_u32(&s_done[0]));
+        }
+        if (!mbar_wait(smem_u32(&s_done[0]), 0) && lane == 0) std::printf("wait expired\n");
+        tc_fence_after();
+        if (warp < 4) {
+            uint32_t v[32];
+            tmem_ld32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + 256, v);
+            tmem_ld_wait();
+            int bad = 0;
+            for (int c = 0; c < 32; ++c) bad += __uint_as_float(v[c]) != static_cast<float>((warp * 32 + lane) * 32 + c);
+            if (bad && blockIdx.x == 0) atomicAdd(mismatches, bad);
+        }
+    } else if (mode == 1) {
+        if (tid == 0) {
+            for (int i = 0; i < count; ++i) tmem_cp_128x256b(tmem + 256 + (i & 15) * 8, a_sw + 2 * (i & 3));
+            umma_commit(smem_u32(&s_done[0]));
+            if (!mbar_wait(smem_u32(&s_done[0]), 0)) std::printf("wait expired\n");
+        }
+    } else if (mode == 2) {
+        if (tid == 0) {
+            for (int i = 0; i < count; ++i) {
+                const uint32_t slot = tmem + 256 + (i & 3) * 32;
+                for (int kq = 0; kq < 4; ++kq) tmem_cp_128x256b(slot + kq * 8, a_sw + 2 * kq);
+                for (int kq = 0; kq < 4; ++kq) umma_tf32_ts(tmem, slot + kq * 8, b_sw + 2 * kq, idesc, 1u);
+            }
+            umma_commit(smem_u32(&s_done[0]));
+            if (!mbar_wait(smem_u32(&s_done[0]), 0)) std::printf("wait expired\n");
+        }
+    } else {
+        if (warp == 0 && lane == 0) {          // copier
+            for (int i = 0; i < count; ++i) {
+                const int sl = i & 3;
+                if (i >= 4 && !mbar_wait(smem_u32(&s_free[sl]), ((i >> 2) - 1) & 1)) { std::printf("copier wait expired\n"); break; }
+                tc_fence_after();
+                for (int kq = 0; kq < 4; ++kq) tmem_cp_128x256b(tmem + 256 + sl * 32 + kq * 8, a_sw + 2 * kq);
+                umma_commit(smem_u32(&s_ready[sl]));
+            }
+        } else if (warp == 1 && lane == 0) {   // MMA issuer
+            for (int i = 0; i < count; ++i) {
+                const int sl = i & 3;
+                if (!mbar_wait(smem_u32(&s_ready[sl]), (i >> 2) & 1)) { std::printf("issuer wait expired\n"); break; }
+                tc_fence_after();
+                for (int kq = 0; kq < 4; ++kq) umma_tf32_ts(tmem, tmem + 256 + sl * 32 + kq * 8, b_sw + 2 * kq, idesc, 1u);
+                umma_commit(smem_u32(&s_free[sl]));
+            }
+            umma_commit(smem_u32(&s_done[0]));
+            if (!mbar_wait(smem_u32(&s_done[0]), 0)) std::printf("wait expired\n");
+        }
+    }
+    __syncthreads();
+    if (tid == 0) cycles[blockIdx.x] = clock64() - t0;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 7) tmem_dealloc(tmem, 512);
+}
+
 template <typename F>
 float best_ms(F f)
 {
@@ -217,6 +311,31 @@ int main()
                             sms * total * 128.0 * n * 8 * 2 / (ms * 1e-3) / 1e12, sms);
             }
         }
+    }
+    {
+        CK(cudaFuncSetAttribute(k_cp, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        int* bad;
+        CK(cudaMalloc(&bad, sizeof(int)));
+        CK(cudaMemset(bad, 0, sizeof(int)));
+        k_cp<<<sms, 256, smem>>>(0, 0, 256, cyc, bad);
+        CK(cudaDeviceSynchronize());
+        int hb = -1;
+        CK(cudaMemcpy(&hb, bad, sizeof(int), cudaMemcpyDeviceToHost));
+        std::printf("cp      layout check: %d mismatching elements of 4096 (row -> lane, 8 consecutive floats -> 8 columns)\n", hb);
+        const int count = 4096;
+        float ms = best_ms([&] { k_cp<<<sms, 256, smem>>>(1, count, 256, cyc, bad); });
+        CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+        std::printf("cp      128x256b copies back to back, one thread : %6.1f cycles per copy (%.1f ns)\n", static_cast<double>(h) / count, ms * 1e6 / count);
+        for (int mode : {2, 3}) {
+            for (int n : {128, 256}) {
+                ms = best_ms([&] { k_cp<<<sms, 256, smem>>>(mode, count, n, cyc, bad); });
+                CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+                std::printf("cp+mma  4 copies + 4 TS MMAs N=%3d per 32-column block, %s : %6.1f cycles per block, %5.0f TFLOP/s over %d SMs\n", n,
+                            mode == 2 ? "one thread " : "two threads", static_cast<double>(h) / count,
+                            sms * static_cast<double>(count) * 4 * 128.0 * n * 8 * 2 / (ms * 1e-3) / 1e12, sms);
+            }
+        }
+        CK(cudaFree(bad));
     }
     CK(cudaFree(cyc));
     return 0;
