@@ -127,7 +127,9 @@ typedef struct {
     int issuers;  /* MMA issuer threads: variant 8: 1-4 (0 = 4); the work item's accumulator columns are cut into
                      that many MMA units where the tile width allows (units of at least 16 columns, none across two
                      tiles), so fewer issuers mean wider MMAs;
-                     variant 4: 1 or 2, each with half of the item's channels (0 = 1) */
+                     variant 4: 1 or 2 (0 = 1); two threads take alternate pipeline stages of a work item, each into an
+                     accumulator of its own that the epilogue adds (the ring then has an even number of stages, and
+                     work items of more than 128 channels have one accumulator buffer instead of two) */
     int ksplit;   /* variant 8: ranges the reduction axis is split into, 1-8 (0 = 1); more than one needs scratch */
     int reserved[8];
 } nm_plan_t;

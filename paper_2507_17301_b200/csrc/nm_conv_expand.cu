@@ -59,7 +59,8 @@ struct ExpandCfg {
     int wres_bytes;   // bytes of the resident slice: all 32-column blocks of bn rows
     int n_sub;        // pipeline stages one work item reduces over: (K / 32) / ksplit / kblk
     int kblk;         // 32-column blocks per stage (1 or 2): one barrier round trip then covers kblk * 4 MMAs
-    int n_iss;        // MMA issuer threads (1 or 2): each owns bn / n_iss accumulator columns and weight rows
+    int n_iss;        // MMA issuer threads (1 or 2): two take alternate pipeline stages of an item, each into an accumulator of its own
+    int n_acc;        // accumulator buffers (of n_iss accumulators each) in tensor memory: 2 when they fit, else 1
     int sub_bytes;    // bytes of one 32-column block inside a stage: activations (+ streamed weights)
     int ksplit;       // K splits (1 = none): a work item covers one of them and stores raw partial sums
     int p_pad;        // pixel blocks * 128: rows of one split in the partial-sum scratch
@@ -154,7 +155,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
     if (tid == 0) {
         for (int i = 0; i < NSTAGE_MAX; ++i) {
             mbar_init(smem_u32(&s_full[i]), 1);   // producer's expect-tx arrival
-            mbar_init(smem_u32(&s_free[i]), cfg.n_iss);   // MMA commits
+            mbar_init(smem_u32(&s_free[i]), 1);   // the commit of the issuer that read the stage
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&s_accfull[i]), cfg.n_iss);   // MMA commits
@@ -260,15 +261,19 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         }
     } else if (warp == 1 || warp == 3) {
         // =========================== MMA issuers ===========================
-        // A thread issues a tcgen05.mma about every 125 cycles whatever its width, and a 128 x 64 x 8 TF32 MMA runs in less:
-        // a plan may share a work item's columns between two issuing threads, each with accumulator columns and
-        // weight rows of its own.  With both operands in shared memory it does not pay (measured: 3-8 % slower on
-        // the layers of 128 channels per item, both threads read the same activation rows), so one thread is the default.
+        // A thread issues a tcgen05.mma about every 124 cycles whatever its width, and a barrier test and a commit per
+        // stage on top of that, while the tensor core completes a 128 x 256 x 8 MMA in 128 cycles and narrower ones
+        // sooner: one thread cannot keep it busy.  A plan may therefore have two issuer threads that take ALTERNATE
+        // stages of a work item, each accumulating into columns of its own (the epilogue adds the two): the reduction
+        // axis is split, not the channels, so both issue full-width MMAs.  A ring slot is released by the one commit of
+        // the thread that read it.  Ownership goes by SLOT (even slots the first thread, odd slots the second; the ring
+        // then has an even number of slots): a wait by phase parity is only right for a waiter that has seen every
+        // earlier use of the slot, and with ownership by position inside the item a thread would skip uses of a slot
+        // at the seams between items (found as a fault on the GPU, reproduced and fixed in a CPU model of the protocol).
         const int iss = warp >> 1;
         if (lane == 0 && iss < cfg.n_iss) {
-            const int mma_n = cfg.bn / cfg.n_iss;
-            const uint32_t idesc = umma_idesc_tf32(BM, mma_n);
-            const uint32_t b_rows = static_cast<uint32_t>(iss * mma_n) * 128u;   // this issuer's weight rows inside a stage
+            const uint32_t idesc = umma_idesc_tf32(BM, cfg.bn);
+            const bool shared_k = cfg.n_iss == 2;
             if (cfg.w_res && !mbar_wait(smem_u32(&s_wres), 0)) *abort_flag = 9;
             RingPos rp;
             uint32_t ab = 0, acc_par = 0;   // accumulator buffer of this item, parity of its current use
@@ -281,31 +286,42 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     break;
                 }
                 tc_fence_after();
-                const uint32_t acc = tmem + ab * cfg.bn + iss * mma_n;
+                const uint32_t acc = tmem + (ab * cfg.n_iss + iss) * cfg.bn;
+                uint32_t started = 0;   // 0 until this thread's first MMA of the item, which overwrites the accumulator
                 for (int c = seg.sb; c < seg.se; ++c) {
+                    if (shared_k && (rp.s & 1) != iss) {   // the other thread's slot
+                        rp.advance(NS);
+                        continue;
+                    }
                     if (!mbar_wait_lone(smem_u32(&s_full[rp.s]), rp.parity)) { *abort_flag = 6; break; }
                     tc_fence_after();
                     const uint32_t a_smem = ring + rp.s * cfg.stage_bytes;
                     uint64_t adesc = umma_desc_k_sw128(a_smem, 1024);
-                    uint64_t bdesc = umma_desc_k_sw128((cfg.w_res ? wres + c * KBLK * cfg.b_bytes : a_smem + SUB_BYTES) + b_rows, 1024);
+                    uint64_t bdesc = umma_desc_k_sw128(cfg.w_res ? wres + c * KBLK * cfg.b_bytes : a_smem + SUB_BYTES, 1024);
                     const uint32_t b_step = KBLK > 1 ? static_cast<uint32_t>(cfg.w_res ? cfg.b_bytes : cfg.sub_bytes) >> 4 : 0u;
 #pragma unroll
                     for (int j = 0; j < KBLK; ++j) {
 #pragma unroll
                         for (int kq = 0; kq < 4; ++kq)
-                            umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (c > seg.sb || j > 0 || kq > 0) ? 1u : 0u);
+                            umma_tf32_ss(acc, adesc + 2 * kq, bdesc + 2 * kq, idesc, (j > 0 || kq > 0) ? 1u : started);
                         if (j + 1 < KBLK) {
                             adesc += static_cast<uint32_t>(cfg.sub_bytes) >> 4;   // next 32-column block (start address field, 16-byte units)
                             bdesc += b_step;
                         }
                     }
+                    started = 1u;
                     umma_commit(smem_u32(&s_free[rp.s]));
                     rp.advance(NS);
                 }
                 if (aborted(abort_flag)) break;
                 umma_commit(smem_u32(&s_accfull[ab]));
-                if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
-                ab ^= 1u;
+                if (cfg.n_acc == 2) {
+                    if (ab == 1) { acc_par ^= 1u; acc_wrapped = true; }
+                    ab ^= 1u;
+                } else {
+                    acc_par ^= 1u;
+                    acc_wrapped = true;
+                }
             }
         }
     } else if (warp >= 4) {
@@ -318,6 +334,7 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
         const uint32_t rx = static_cast<uint32_t>(lane & 7);
         const int n_blk = cfg.bn / 32;
         uint32_t nb = 0, ti = 0;
+        uint32_t stage_count = 0;   // stages of all earlier pieces of this CTA
         // balanced mode: this CTA's partial-sum slot (128 rows x bn) and its warps' flags, in the handle's scratch
         const uint32_t units = static_cast<uint32_t>(cfg.n_work) * static_cast<uint32_t>(cfg.n_sub);
         const size_t slot_floats = static_cast<size_t>(BM) * cfg.bn;
@@ -335,7 +352,13 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
             const uint32_t rest = work / static_cast<uint32_t>(cfg.n_slices);
             const int ks = static_cast<int>(rest % static_cast<uint32_t>(cfg.ksplit));
             const uint32_t pix0 = (rest / static_cast<uint32_t>(cfg.ksplit)) * BM;
-            const int ab = static_cast<int>(ti & 1u);
+            const int ab = cfg.n_acc == 2 ? static_cast<int>(ti & 1u) : 0;
+            // two issuers: stages went to them by ring slot, i.e. by the parity of the running stage count; a piece of
+            // one stage is in the accumulator of that stage's owner, a longer one in both
+            const uint32_t piece_first = stage_count;
+            stage_count += static_cast<uint32_t>(seg.se - seg.sb);
+            const bool two_acc = cfg.n_iss == 2 && seg.se - seg.sb >= 2;
+            const uint32_t acc_first = (cfg.n_iss == 2 && seg.se - seg.sb == 1) ? (piece_first & 1u) : 0u;
             // the shortcut input does not depend on the accumulator: its first box is requested before the
             // wait for the main loop, every later box while the one before it is being stored
             const long long box_pix = static_cast<long long>(pix0) + q * 32;
@@ -374,14 +397,22 @@ k_conv_expand(const ConvParams p, const ExpandCfg cfg, const __grid_constant__ C
                     ahead = true;
                 }
             }
-            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (ti >> 1) & 1u);
+            const bool ok = aborted(abort_flag) || mbar_wait(smem_u32(&s_accfull[ab]), (cfg.n_acc == 2 ? (ti >> 1) : ti) & 1u);
             if (!__all_sync(0xFFFFFFFFu, ok)) *abort_flag = 8;
             if (__any_sync(0xFFFFFFFFu, aborted(abort_flag))) break;
             tc_fence_after();
             for (int blk = half; blk < n_blk; blk += 2, ++nb) {
                 uint32_t v[32];
-                tmem_ld32(tmem + lane_addr + ab * cfg.bn + blk * 32, v);
-                tmem_ld_wait();
+                tmem_ld32(tmem + lane_addr + (ab * cfg.n_iss + acc_first) * cfg.bn + blk * 32, v);
+                if (two_acc) {
+                    uint32_t v2[32];
+                    tmem_ld32(tmem + lane_addr + (ab * cfg.n_iss + 1) * cfg.bn + blk * 32, v2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(v2[e]));
+                } else {
+                    tmem_ld_wait();
+                }
                 if (blk + 2 >= n_blk) {
                     tc_fence_before();
                     __syncwarp();
@@ -578,10 +609,12 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     if (kblk > 2 || blk32 % kblk != 0) return false;
     cfg->kblk = kblk;
     cfg->n_sub = blk32 / kblk;
-    // one issuer thread unless the plan asks for two (halves of whole 8-row swizzle atoms, MMA widths multiples of 16)
+    // one issuer thread unless the plan asks for two (alternate stages, an accumulator each; one accumulator buffer
+    // instead of two when both pairs do not fit the 512 columns)
     const int n_iss = plan && plan->issuers > 0 ? plan->issuers : 1;
-    if (n_iss < 1 || n_iss > 2 || bn % (16 * n_iss) != 0) return false;
+    if (n_iss < 1 || n_iss > 2) return false;
     cfg->n_iss = n_iss;
+    cfg->n_acc = 2 * n_iss * bn <= 512 ? 2 : 1;
     cfg->p_pad = static_cast<int>(((p.pixels + BM - 1) / BM) * BM);
     if (splits > 1 && (!p.splitk || p.splitk_bytes < static_cast<size_t>(splits) * cfg->p_pad * p.c_out * sizeof(float) ||
                        static_cast<long long>(splits) * cfg->p_pad >= (1ll << 31)))
@@ -604,8 +637,10 @@ bool make_cfg(const ConvParams& p, const nm_plan_t* plan, ExpandCfg* cfg)
     if (stages > NSTAGE_MAX) return false;
     if (plan && plan->stages > 0) {
         if (stages * cfg->stage_bytes > budget) return false;
+        if (n_iss == 2 && stages % 2 != 0) return false;   // two issuers own alternate ring slots
     } else {
         while (stages > 2 && stages * cfg->stage_bytes > budget) --stages;
+        if (n_iss == 2) stages &= ~1;
         if (stages * cfg->stage_bytes > budget) return false;
     }
     cfg->stages = stages;

@@ -245,6 +245,91 @@ __global__ void __launch_bounds__(256, 1) k_cp(int mode, int count, int n, long 
     if (warp == 7) tmem_dealloc(tmem, 512);
 }
 
+// The main loop of a pipelined kernel without its loads: one thread issues `group` SS MMAs 128 x 256 x 8 per ring stage
+// (four stages of 48 KB: 16 KB of A, 32 KB of B), then a tcgen05.commit to the stage's barrier; with `wait` it first tests
+// another stage's barrier (non-blocking), as an issuer does before it reads a stage.
+__global__ void __launch_bounds__(256, 1) k_mma_loop(int stages_total, int group, int wait, long long* cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem;
+    __shared__ uint64_t s_done, s_ring[4];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < 4 * 12288; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw)[i] = 0;
+    if (warp == 7) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (tid == 0) {
+        mbar_init(smem_u32(&s_done), 1);
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&s_ring[i]), 1);
+        mbar_fence_init();
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const long long t0 = clock64();
+    if (tid == 0) {
+        const uint32_t idesc = umma_idesc_tf32(128, 256);
+        uint32_t sink = 0;
+        // wait = 2: the commits of two stages are issued together after the second stage's MMAs
+        for (int st = 0; st < stages_total; ++st) {
+            const uint32_t stage = base + (st & 3) * 49152;
+            if (wait) sink += mbar_test_wait(smem_u32(&s_ring[(st + 2) & 3]), (st >> 2) & 1) ? 1u : 0u;
+            const uint64_t adesc = umma_desc_k_sw128(stage, 1024), bdesc = umma_desc_k_sw128(stage + 16384, 1024);
+            for (int i = 0; i < group; ++i) umma_tf32_ss(tmem, adesc + 2 * (i & 3), bdesc + 2 * (i & 3), idesc, 1u);
+            if (wait != 2) {
+                umma_commit(smem_u32(&s_ring[st & 3]));
+            } else if (st & 1) {
+                umma_commit(smem_u32(&s_ring[(st - 1) & 3]));
+                umma_commit(smem_u32(&s_ring[st & 3]));
+            }
+        }
+        umma_commit(smem_u32(&s_done));
+        if (!mbar_wait(smem_u32(&s_done), 0)) std::printf("wait expired\n");
+        if (sink == 0xFFFFFFFFu) std::printf("%u\n", sink);
+    }
+    __syncthreads();
+    if (tid == 0) cycles[blockIdx.x] = clock64() - t0;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 7) tmem_dealloc(tmem, 512);
+}
+
+// One buffer pair read over and over: does the placement of the two operands in shared memory matter?  A (16 KB) at
+// `a_off`, B (32 KB) at `b_off` from a 1024-byte-aligned base; `group` MMAs cycle over the four K-steps of the tile.
+__global__ void __launch_bounds__(256, 1) k_mma_place(int count, uint32_t a_off, uint32_t b_off, int ksteps, long long* cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t s_tmem;
+    __shared__ uint64_t s_done;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < 49152; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw)[i] = 0;
+    if (warp == 7) tmem_alloc(smem_u32(&s_tmem), 512);
+    if (tid == 0) { mbar_init(smem_u32(&s_done), 1); mbar_fence_init(); }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const long long t0 = clock64();
+    if (tid == 0) {
+        const uint32_t idesc = umma_idesc_tf32(128, 256);
+        const uint64_t adesc = umma_desc_k_sw128(base + a_off, 1024), bdesc = umma_desc_k_sw128(base + b_off, 1024);
+        for (int i = 0; i < count; ++i) {
+            const int kq = ksteps == 4 ? (i & 3) : 0;
+            umma_tf32_ss(tmem, adesc + 2 * kq, bdesc + 2 * kq, idesc, 1u);
+        }
+        umma_commit(smem_u32(&s_done));
+        if (!mbar_wait(smem_u32(&s_done), 0)) std::printf("wait expired\n");
+    }
+    __syncthreads();
+    if (tid == 0) cycles[blockIdx.x] = clock64() - t0;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 7) tmem_dealloc(tmem, 512);
+}
+
 template <typename F>
 float best_ms(F f)
 {
@@ -309,6 +394,32 @@ int main()
                 std::printf("mma     %s N=%3d issuers=%d : %6.1f cycles per MMA, %6.1f ns, %5.0f TFLOP/s over %d SMs\n", names[ss], n,
                             issuers, static_cast<double>(h) / total, ms * 1e6 / total,
                             sms * total * 128.0 * n * 8 * 2 / (ms * 1e-3) / 1e12, sms);
+            }
+        }
+    }
+    {
+        const size_t big = 200 * 1024;
+        CK(cudaFuncSetAttribute(k_mma_loop, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(big)));
+        for (int group : {4, 8, 16}) {
+            for (int wait : {0, 1, 2}) {
+                const int total = 8192 / group;
+                const float ms = best_ms([&] { k_mma_loop<<<sms, 256, big>>>(total, group, wait, cyc); });
+                CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+                std::printf("loop    SS N=256, %2d MMAs per stage, commit per stage%s : %6.1f cycles per MMA (%.1f ns)\n", group,
+                            wait == 2 ? ", barrier test before, commits in pairs" : wait ? ", barrier test before" : "", static_cast<double>(h) / 8192, ms * 1e6 / 8192);
+            }
+        }
+    }
+    {
+        const size_t big = 200 * 1024;
+        CK(cudaFuncSetAttribute(k_mma_place, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(big)));
+        const uint32_t offs[][2] = {{32768, 0}, {0, 16384}, {0, 32768}, {49152, 65536}, {0, 49152}, {1024, 32768}, {0, 98304}, {131072, 0}};
+        for (const auto& o : offs) {
+            for (int ksteps : {4, 1}) {
+                const float ms = best_ms([&] { k_mma_place<<<sms, 256, big>>>(8192, o[0], o[1], ksteps, cyc); });
+                CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+                std::printf("place   SS N=256, A at %6u, B at %6u, %s : %6.1f cycles per MMA (%.1f ns)\n", o[0], o[1],
+                            ksteps == 4 ? "four K-steps in turn" : "one K-step repeated ", static_cast<double>(h) / 8192, ms * 1e6 / 8192);
             }
         }
     }

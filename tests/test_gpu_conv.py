@@ -36,9 +36,12 @@ def _plans(nm, s):
         p = nm.nm_plan_t()
         p.variant, p.bn, p.stages, p.split, p.kblk = 4, bn, stages, split, kblk
         out.append(p)
-    for bn, issuers in ((0, 1), (128, 1), (64, 2), (256, 2), (32, 2)):   # one and two MMA issuer threads
+    # one and two MMA issuer threads (two: alternate stages, an accumulator each; one accumulator buffer at 256 channels),
+    # with weights resident / streamed, one and two blocks per stage, a two-stage ring
+    for bn, issuers, split, kblk, stages in ((0, 1, 0, 0, 0), (128, 1, 0, 0, 0), (64, 2, 0, 0, 0), (256, 2, 0, 0, 0), (32, 2, 0, 0, 0),
+                                             (0, 2, 1, 2, 0), (256, 2, 1, 1, 2), (128, 2, 1, 2, 2), (64, 2, 1, 1, 4)):
         p = nm.nm_plan_t()
-        p.variant, p.bn, p.issuers = 4, bn, issuers
+        p.variant, p.bn, p.issuers, p.split, p.kblk, p.stages = 4, bn, issuers, split, kblk, stages
         out.append(p)
     p = nm.nm_plan_t()
     p.variant = 5                                     # row-run kernel
@@ -328,6 +331,7 @@ def test_split_k_plans(nm, integer):
             plan = nm.nm_plan_t()
             plan.variant, plan.bn, plan.split = 4, bn, splits
             plan.kblk = 2 if bn == 64 else 0                  # K / 32 / splits = 36, 24, 18: two blocks per stage fit
+            plan.issuers = 2 if splits == 3 else 0            # one of the splits with two issuer threads
             for _ in range(2):                                # twice: the scratch is reused
                 y = nm.nm_conv2d(hnd, xd, s.kh, s.kw, s.stride, s.pad, s.dil, bd, s.relu, plan=plan)
             nm.nm_weights_check(hnd)
@@ -359,11 +363,11 @@ def test_balanced_plans(nm, s, integer):
     hnd = nm.nm_prune(w.cuda(), s.n_keep, s.m_group, s.tile_t)
     xd, bd = x.cuda(), b.cuda()
     ran = 0
-    for bn, kblk, stages in ((64, 0, 0), (128, 2, 0), (32, 1, 2), (256, 0, 0)):
+    for bn, kblk, stages, issuers in ((64, 0, 0, 0), (128, 2, 0, 0), (32, 1, 2, 0), (256, 0, 0, 0), (256, 0, 0, 2), (128, 2, 0, 2), (64, 1, 2, 2)):
         if s.c_out % bn:
             continue
         plan = nm.nm_plan_t()
-        plan.variant, plan.bn, plan.split, plan.kblk, plan.stages = 4, bn, -1, kblk, stages
+        plan.variant, plan.bn, plan.split, plan.kblk, plan.stages, plan.issuers = 4, bn, -1, kblk, stages, issuers
         need = nm.nm_plan_scratch_bytes(hnd, xd.shape, s.stride, s.pad, s.dil, plan)
         assert need >= 128 * bn * 4
         nm.nm_weights_reserve(hnd, need)

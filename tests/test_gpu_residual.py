@@ -43,9 +43,9 @@ def test_residual_epilogue(nm, s, integer):
     xd, bd, rd = x.cuda(), b.cuda(), res.cuda()
     nm.nm_autotune(hnd, xd, s.stride, s.pad, s.dil, bd, True, kh=s.kh, kw=s.kw)    # reserves split-K scratch if any
     plans = _plans(nm, s)
-    for splits, kblk in ((2, 0), (3, 0), (-1, 0), (-1, 2)):   # split-K, and balanced ranges (need the tuner's scratch)
+    for splits, kblk, issuers in ((2, 0, 0), (3, 0, 0), (-1, 0, 0), (-1, 2, 0), (2, 0, 2), (-1, 0, 2)):   # split-K, and balanced ranges (need the tuner's scratch)
         p = nm.nm_plan_t()
-        p.variant, p.bn, p.split, p.kblk = 4, 64, splits, kblk
+        p.variant, p.bn, p.split, p.kblk, p.issuers = 4, 64, splits, kblk, issuers
         plans.append(p)
     ran = set()
     for plan in plans:
