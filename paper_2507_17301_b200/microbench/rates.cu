@@ -6,6 +6,8 @@
 //            loaded from shared memory), byte masks (one byte per select, widened with a byte permute).
 //   mma      TF32 tcgen05.mma of shape 128 x N x 8 issued back to back by 1, 2 or 4 threads (each with accumulator
 //            columns of its own), A from tensor memory (TS) or from shared memory (SS).
+//   intake   bytes per cycle an SM takes in from L2: bulk copies of 32 KB, tiled TMA loads of 128 rows x 128 bytes (swizzled), or
+//            one of each per stage, four stages in flight, every SM reading its own 1 MB window of a buffer that fits the L2.
 //   cp       tcgen05.cp of an operand tile from shared to tensor memory: layout check, issue rate, and the rate of
 //            the pattern "four copies, four TS MMAs" per 32-column block from one and from two threads.
 //
@@ -15,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include "../csrc/nm_ptx.cuh"
+#include "../csrc/nm_tmap.cuh"
 using namespace nmk;
 
 #define CK(x)                                                                                  \
@@ -330,6 +333,39 @@ __global__ void __launch_bounds__(256, 1) k_mma_place(int count, uint32_t a_off,
     if (warp == 7) tmem_dealloc(tmem, 512);
 }
 
+// MODE 0: one 32 KB bulk copy per stage; 1: one tiled TMA load of 128 rows x 128 bytes (16 KB) per stage; 2: both (48 KB, the
+// expanded-operand kernel's stage).  One thread keeps four stages in flight; nothing consumes the data.
+__global__ void __launch_bounds__(128, 1) k_intake(int mode, int stages_total, const float* src, const __grid_constant__ CUtensorMap tm,
+                                                  long long* cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t s_full[4];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&s_full[i]), 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    const long long t0 = clock64();
+    if (threadIdx.x == 0) {
+        const uint32_t tx = mode == 0 ? 32768u : mode == 1 ? 16384u : 49152u;
+        const float* mine = src + static_cast<size_t>(blockIdx.x) * 262144;       // 1 MB window per SM
+        for (int st = 0; st < stages_total + 4; ++st) {
+            const int sl = st & 3;
+            if (st >= 4 && !mbar_wait(smem_u32(&s_full[sl]), ((st >> 2) - 1) & 1)) { std::printf("wait expired\n"); break; }
+            if (st < stages_total) {
+                const uint32_t dst = base + sl * 49152, bar = smem_u32(&s_full[sl]);
+                mbar_arrive_expect_tx(bar, tx);
+                const int piece = st & 7;                                        // 8 pieces of 64 KB: 512 KB per SM, 74 MB in all (fits the L2)
+                if (mode != 1) bulk_load_1d(dst + 16384, mine + piece * 16384, 32768, bar);
+                if (mode != 0) tma_load_2d(dst, &tm, bar, (st & 7) * 32, static_cast<int>(blockIdx.x) * 1024 + (piece & 7) * 128);
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) cycles[blockIdx.x] = clock64() - t0;
+}
+
 template <typename F>
 float best_ms(F f)
 {
@@ -422,6 +458,34 @@ int main()
                             ksteps == 4 ? "four K-steps in turn" : "one K-step repeated ", static_cast<double>(h) / 8192, ms * 1e6 / 8192);
             }
         }
+    }
+    if (nmtm::available()) {
+        // a [148 * 1024 rows][256 floats] buffer, of which every SM re-reads 512 KB of its own 1 MB (74 MB in all: L2 hits)
+        const size_t rows = static_cast<size_t>(sms) * 1024, cols = 256;
+        float* buf;
+        CK(cudaMalloc(&buf, rows * cols * sizeof(float)));
+        CK(cudaMemset(buf, 0, rows * cols * sizeof(float)));
+        alignas(64) CUtensorMap tm;
+        const cuuint64_t dims[2] = {cols, rows};
+        const cuuint64_t strides[1] = {cols * sizeof(float)};
+        const cuuint32_t box[2] = {32, 128}, es[2] = {1, 1};
+        if (nmtm::encoders().tiled(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, buf, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS) {
+            const size_t big = 200 * 1024;
+            CK(cudaFuncSetAttribute(k_intake, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(big)));
+            const char* what[3] = {"32 KB bulk copy per stage        ", "16 KB tiled load per stage       ", "bulk copy + tiled load (48 KB)   "};
+            const double bytes[3] = {32768, 16384, 49152};
+            for (int mode = 0; mode < 3; ++mode) {
+                const int total = 2048;
+                const float ms = best_ms([&] { k_intake<<<sms, 128, big>>>(mode, total, buf, tm, cyc); });
+                CK(cudaMemcpy(&h, cyc, sizeof(h), cudaMemcpyDeviceToHost));
+                std::printf("intake  %s: %6.1f cycles per stage, %5.1f bytes per cycle and SM, %5.2f TB/s over %d SMs\n", what[mode],
+                            static_cast<double>(h) / total, bytes[mode] * total / static_cast<double>(h),
+                            sms * bytes[mode] * total / (ms * 1e-3) / 1e12, sms);
+            }
+        }
+        CK(cudaFree(buf));
     }
     {
         CK(cudaFuncSetAttribute(k_cp, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
